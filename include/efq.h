@@ -1,0 +1,157 @@
+/*
+ * efq.h - C ABI of the B200 (sm_100a) EFQ-Softmax library.
+ *
+ * EFQ-Softmax replaces the exp-then-quantize producer of a block-scaled FP4 attention
+ * forward by direct generation of the low-bit probability operand: per 32-key
+ * microscaling block an exponent-only E8M0 scale taken from the block's largest shifted
+ * score, and per element a nonnegative E2M1 code from one affine rule.  The same operand
+ * feeds the numerator P~V and the denominator P~1; the online-softmax recurrence around
+ * it is unchanged.
+ *
+ * Conventions for every entry point
+ *   - Pointers are DEVICE pointers unless the parameter name ends in _host.
+ *   - The library never allocates or frees device memory on these paths; the caller owns
+ *     every buffer, including the workspace, for the duration of the stream work.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Launches
+ *     are asynchronous; a returned EFQ_OK means "validated and enqueued".
+ *   - Errors are return codes; nothing aborts or traps.  Device-side waits are bounded and
+ *     report through the status word read by efq_poll_status().
+ *   - Packed E2M1 codes: element 2u sits in bits 0-3 of byte u, element 2u+1 in bits 4-7.
+ *     Probability codes are nonnegative (bit 3 of every nibble is 0).
+ *   - E8M0 scale byte b means the power of two 2^(b-127).
+ *   - Microscaling block: 32 consecutive keys (columns), aligned to absolute index.
+ */
+#ifndef EFQ_H_
+#define EFQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    EFQ_OK = 0,
+    EFQ_ERR_INVALID_ARG = 1,    /* null pointer, non-positive size, non-finite parameter, Hq % Hkv != 0 */
+    EFQ_ERR_UNSUPPORTED = 2,    /* d != 128, kv_tile not supported, variant not built */
+    EFQ_ERR_ALIGNMENT = 3,      /* a pointer or leading dimension breaks the stated alignment */
+    EFQ_ERR_WORKSPACE = 4,      /* workspace pointer null or smaller than efq_attention_workspace_bytes() */
+    EFQ_ERR_ARCH = 5,           /* current device is not compute capability 10.x */
+    EFQ_ERR_CUDA = 6,           /* a CUDA runtime/driver call failed (launch, copy, descriptor encode) */
+    EFQ_ERR_DEVICE_TIMEOUT = 7  /* a bounded device-side wait expired; the output is invalid */
+} efq_status_t;
+
+/* Parameters of the affine code rule c = clip_[0,7](floor((z - tau) h) + 1)
+ * (Eq. d8-index).  (tau, h) are global, fixed after calibration; the operating points
+ * printed in the paper are EFQ-Mean (-3.06, 2.30), EFQ-MMLU (-2.90, 2.00) and
+ * EFQ-Balance (-2.10, 2.70).  Passing NULL for a params pointer selects EFQ-Mean,
+ * variant 0, kv_tile 128. */
+typedef struct {
+    float tau;
+    float h;          /* > 0 */
+    int32_t variant;  /* 0 = affine rule (Eq. d8-index); 1 = 16-level LUT variant (Sec. 3.4) */
+    int32_t kv_tile;  /* Bc, keys per online-softmax step; 0 = default (128).  The shifted score uses the
+                         running row maximum that includes the current KV block (Algorithm 2, steps 2-3),
+                         so codes depend on this width.  Must be 128 in this build. */
+} efq_params_t;
+
+/* Optional debug dump of the fused forward for one head and a range of query rows.
+ * Any pointer may be NULL.  Row r of each buffer is query row q_begin + r.
+ *   raw_scores  fp32 [q_end-q_begin, Sk]            Q^ K^T before the softmax scale; masked keys hold -inf
+ *   row_max     fp32 [q_end-q_begin, ceil(Sk/Bc)]   scaled running maximum m_s used for each KV tile
+ *   codes       u8   [q_end-q_begin, ceil(Sk/32)*16] packed probability codes (linear order)
+ *   scales      u8   [q_end-q_begin, ceil(Sk/32)]   E8M0 bytes */
+typedef struct {
+    float* raw_scores;
+    float* row_max;
+    uint8_t* codes;
+    uint8_t* scales;
+    int32_t batch;
+    int32_t head;
+    int64_t q_begin;
+    int64_t q_end;
+} efq_debug_t;
+
+/* Probability-generation stage on a score matrix (kernel interface of Sec. 4.3:
+ * (x, B, tau, h) -> (Q_P, s_P); Algorithm 1 applied to every 32-column block).
+ *   scores   fp32 [rows, ld], 16-byte aligned, ld >= cols and ld % 4 == 0; masked entries = -inf
+ *   row_max  fp32 [rows], the row maximum in scaled units: the shifted score is
+ *            x = score_scale * scores - row_max
+ *   codes    u8 [rows, ceil(cols/32)*16], 16-byte aligned; positions past `cols` in the last
+ *            block get code 0
+ *   scales   u8 [rows, ceil(cols/32)]; a block with no finite entry gets byte 0 and zero codes
+ * Returns INVALID_ARG for null pointers, rows/cols < 0, h <= 0 or non-finite parameters,
+ * ALIGNMENT as stated above.  rows == 0 or cols == 0 is a valid no-op. */
+efq_status_t efq_probgen(const float* scores, int64_t ld, const float* row_max, int64_t rows, int64_t cols,
+                         float score_scale, const efq_params_t* params, uint8_t* codes, uint8_t* scales,
+                         void* stream);
+
+/* The conventional producer on the same interface (Eq. post-softmax-path):
+ * p = exp(x) in FP32, per block e = floor(log2 max p) - 2 (scale_mode 0, block maximum in
+ * [4, 8)) or e = ceil(log2(max p / 6)) (scale_mode 1, block maximum in (3, 6]),
+ * q = round-to-nearest-even E2M1 of p 2^-e, saturating.  Same layouts and errors. */
+efq_status_t exp_then_quantize_probgen(const float* scores, int64_t ld, const float* row_max, int64_t rows,
+                                       int64_t cols, float score_scale, int scale_mode, uint8_t* codes,
+                                       uint8_t* scales, void* stream);
+
+/* Bytes of caller-owned device workspace the fused forward needs for a problem shape
+ * (MXFP4 copies of Q, K, V with their scale tensors, tensor-map descriptors, status word).
+ * Returns 0 for an unsupported shape. */
+size_t efq_attention_workspace_bytes(int B, int Hq, int Hkv, int64_t Sq, int64_t Sk, int d);
+
+/* Fused block-scaled FP4 attention forward with EFQ probability generation
+ * (Algorithm 2 looped over KV tiles; Algorithm 1 per microscaling block).
+ *   q        bf16 [B, Hq, Sq, d] contiguous, 16-byte aligned
+ *   k, v     bf16 [B, Hkv, Sk, d] contiguous, 16-byte aligned; query head h reads KV head h / (Hq/Hkv)
+ *   o        fp32 [B, Hq, Sq, d]
+ *   causal   nonzero: query i sees keys t <= i + Sk - Sq (bottom-right aligned)
+ *   softmax_scale  <= 0 selects 1/sqrt(d)
+ *   workspace  device, 1024-byte aligned, >= efq_attention_workspace_bytes(...)
+ * Q, K (blocks of 32 along d) and V (blocks of 32 along keys) are first quantised to MXFP4
+ * (shared exponent floor(log2 amax) - 2, round-to-nearest-even, saturating); a query row with
+ * no visible key yields zeros.  d must be 128 (UNSUPPORTED otherwise). */
+efq_status_t efq_attention_fwd(const void* q, const void* k, const void* v, float* o, int B, int Hq, int Hkv,
+                               int64_t Sq, int64_t Sk, int d, int causal, float softmax_scale,
+                               const efq_params_t* params, void* workspace, size_t workspace_bytes,
+                               const efq_debug_t* debug, void* stream);
+
+/* The MXFP4 comparison path: identical pipeline, the producer replaced by exp-then-quantize
+ * (scale_mode as in exp_then_quantize_probgen).  The denominator comes from the same
+ * quantised operand as the numerator. */
+efq_status_t exp_then_quantize_attention_fwd(const void* q, const void* k, const void* v, float* o, int B,
+                                             int Hq, int Hkv, int64_t Sq, int64_t Sk, int d, int causal,
+                                             float softmax_scale, int scale_mode, void* workspace,
+                                             size_t workspace_bytes, const efq_debug_t* debug, void* stream);
+
+/* End-to-end form with HOST inputs and output: copies q/k/v from (preferably pinned) host
+ * memory into caller-owned device staging buffers, runs the forward selected by `producer`
+ * (0 = EFQ, 1 = exp-then-quantize scale4, 2 = exp-then-quantize scale6), copies o back, all on
+ * `stream`.  q_dev/k_dev/v_dev/o_dev are device buffers of the same sizes as the host ones. */
+efq_status_t efq_attention_fwd_host(const void* q_host, const void* k_host, const void* v_host, float* o_host,
+                                    void* q_dev, void* k_dev, void* v_dev, float* o_dev, int B, int Hq, int Hkv,
+                                    int64_t Sq, int64_t Sk, int d, int causal, float softmax_scale, int producer,
+                                    const efq_params_t* params, void* workspace, size_t workspace_bytes,
+                                    void* stream);
+
+/* Synchronises `stream` and returns the device-side status word of the last forward that
+ * used `workspace` (EFQ_OK, or EFQ_ERR_DEVICE_TIMEOUT if a bounded wait expired), or
+ * EFQ_ERR_CUDA if the stream reports an error. */
+efq_status_t efq_poll_status(void* workspace, void* stream);
+
+/* Dense FP4 tensor-pipe microbenchmark: `iters` back-to-back 128x256x64 block-scaled E2M1 MMAs
+ * per CTA on operands resident in shared memory, one CTA per SM.  Writes nothing but a
+ * checksum word per CTA to `sink` (u32 [num_ctas]).  Used to measure the MMA-only FP4 rate
+ * that the fused forward's tensor-pipe fraction is quoted against.  Returns the FLOPs per
+ * launch through *flops. */
+efq_status_t efq_fp4_mma_peak_probe(uint32_t* sink, int num_ctas, int iters, double* flops, void* stream);
+
+const char* efq_status_string(efq_status_t status);
+
+/* Library build tag, e.g. "efq-b200 sm_100a". */
+const char* efq_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EFQ_H_ */

@@ -1,0 +1,94 @@
+// Shared device/host helpers of the EFQ-Softmax B200 library (sm_100a only).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+
+#include "efq.h"
+
+namespace efq {
+
+constexpr int kMxBlock = 32;  // keys per microscaling block
+
+// Constants of the FP32 code rule, derived on the host in double and rounded once.
+// With x = sigma*r - m_s, k the block's scale exponent and z = x - k ln2 - ln6 (Eq. z-def):
+//   (z - tau) h + 1  =  r*(sigma h) - h m_s - k (h ln2) + (1 - h (ln6 + tau))
+struct ProducerConsts {
+    float A;      // sigma * h
+    float HL2;    // h * ln 2
+    float C1;     // 1 - h * (ln 6 + tau)
+    float h;
+    float sigma;
+    float LOG2E;  // 1 / ln 2
+    float L2_29;  // log2(2/9), the constant of the scale rule (Eq. k-rule)
+};
+
+inline ProducerConsts make_producer_consts(float sigma, float tau, float h)
+{
+    ProducerConsts c;
+    const double ln2 = 0.693147180559945309417232121458, ln6 = 1.79175946922805500081247735838;
+    c.A = static_cast<float>(static_cast<double>(sigma) * static_cast<double>(h));
+    c.HL2 = static_cast<float>(static_cast<double>(h) * ln2);
+    c.C1 = static_cast<float>(1.0 - static_cast<double>(h) * (ln6 + static_cast<double>(tau)));
+    c.h = h;
+    c.sigma = sigma;
+    c.LOG2E = static_cast<float>(1.0 / ln2);
+    c.L2_29 = static_cast<float>(log(2.0 / 9.0) / ln2);
+    return c;
+}
+
+#ifdef __CUDACC__
+
+// Per-block part of Algorithm 1 (steps 1-3): from the block's largest raw score and the
+// row maximum m_s (scaled units) to the E8M0 byte and the additive term of the code rule.
+// Separate mul and sub (never contracted) so the result equals the reference FP32 order.
+struct BlockScale {
+    float Bb;       // additive term: v_t = fma(r_t, A, Bb)
+    uint32_t byte;  // k_b + 127, or 0 for a block with no finite score
+    bool live;
+};
+
+__device__ __forceinline__ BlockScale efq_block_scale(float rmax, float m_s, const ProducerConsts& K)
+{
+    BlockScale s;
+    s.live = rmax != -INFINITY;
+    float Mb = __fsub_rn(__fmul_rn(K.sigma, rmax), m_s);
+    float kf = floorf(__fmaf_rn(Mb, K.LOG2E, K.L2_29));
+    kf = fminf(fmaxf(kf, -127.0f), 127.0f);
+    s.Bb = __fmaf_rn(-K.h, m_s, __fmaf_rn(-K.HL2, kf, K.C1));
+    s.byte = s.live ? static_cast<uint32_t>(static_cast<int>(kf) + 127) : 0u;
+    return s;
+}
+
+// Per-element part (steps 5-7): affine index, clip to [0,7], floor; the result is the
+// 4-bit E2M1 pattern itself (Eq. d8-index).  -inf (masked) maps to 0.
+__device__ __forceinline__ uint32_t efq_code(float r, float A, float Bb)
+{
+    float v = __fmaf_rn(r, A, Bb);
+    v = fminf(fmaxf(v, 0.0f), 7.0f);
+    return static_cast<uint32_t>(__float2int_rd(v));
+}
+
+__device__ __forceinline__ float ex2_approx(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Two floats -> one byte of E2M1 (round-to-nearest-even, saturating); `lo` lands in bits 0-3.
+__device__ __forceinline__ uint32_t cvt_e2m1x2(float lo, float hi)
+{
+    uint16_t out;
+    asm("{ .reg .b8 t;\n"
+        "  cvt.rn.satfinite.e2m1x2.f32 t, %2, %1;\n"
+        "  mov.b16 %0, {t, 0}; }\n"
+        : "=h"(out)
+        : "f"(lo), "f"(hi));
+    return out;
+}
+
+#endif  // __CUDACC__
+
+}  // namespace efq

@@ -1,0 +1,179 @@
+// Standalone probability-generation stage (kernel interface of Sec. 4.3): a streaming,
+// HBM-bound pass over an fp32 score matrix that emits packed E2M1 codes and one E8M0
+// byte per 32-column microscaling block.  Two producers share the data movement:
+//   EFQ  - Algorithm 1: exponent-only scale from the block maximum + one affine rule, no exp;
+//   ETQ  - exp -> FP32 probabilities -> block abs-max -> scale -> round to E2M1.
+//
+// Data movement: one warp owns 1024 consecutive columns of a row (32 blocks).  Lane l in
+// pass i loads the float4 at element (i*32 + l)*4, so every load instruction covers 512
+// contiguous bytes; a microscaling block is spread over 8 adjacent lanes and its maximum
+// is a 3-step butterfly.  Each lane then holds 4 codes (16 bits) per pass; the 16-bit
+// pieces of a pass are contiguous in the packed output (64 bytes per warp per pass).
+// Algorithmic traffic: 4 B/element in, 0.5 B/element + 1 B/32 elements out.
+#include "efq_common.cuh"
+
+namespace efq {
+
+enum Producer : int { kEfq = 0, kEtq4 = 1, kEtq6 = 2 };
+
+constexpr int kSegCols = 1024;       // columns per warp task
+constexpr int kWarpsPerCta = 8;
+
+template <int PRODUCER>
+__device__ __forceinline__ void produce_block(const float (&r)[4], float m_s, const ProducerConsts& K,
+                                              uint32_t& code16, uint32_t& byte)
+{
+    if (PRODUCER == kEfq) {
+        float rmax = fmaxf(fmaxf(r[0], r[1]), fmaxf(r[2], r[3]));
+        rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, 1));
+        rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, 2));
+        rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, 4));
+        BlockScale s = efq_block_scale(rmax, m_s, K);
+        uint32_t c = efq_code(r[0], K.A, s.Bb) | (efq_code(r[1], K.A, s.Bb) << 4) |
+                     (efq_code(r[2], K.A, s.Bb) << 8) | (efq_code(r[3], K.A, s.Bb) << 12);
+        code16 = s.live ? c : 0u;
+        byte = s.byte;
+    } else {
+        float p[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            float x = __fsub_rn(__fmul_rn(K.sigma, r[u]), m_s);
+            p[u] = ex2_approx(__fmul_rn(x, K.LOG2E));   // exp(-inf) = 0 covers masked entries
+        }
+        float amax = fmaxf(fmaxf(p[0], p[1]), fmaxf(p[2], p[3]));
+        amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+        amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+        amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 4));
+        if (amax == 0.0f) {
+            code16 = 0u;
+            byte = 0u;
+            return;
+        }
+        uint32_t bits = __float_as_uint(amax);
+        int E = static_cast<int>((bits >> 23) & 0xffu) - 127;
+        int e;
+        if (PRODUCER == kEtq4) {
+            e = E - 2;                                   // maximum lands in [4, 8)
+        } else {
+            e = (bits & 0x7fffffu) > 0x400000u ? E - 1 : E - 2;   // smallest e with amax <= 6 * 2^e
+        }
+        e = max(e, -127);
+        // 2^-e as a float: e is in [-127, 125], so the exponent field 127 - e is in [2, 254].
+        const float s = __uint_as_float(static_cast<uint32_t>(127 - e) << 23);
+        uint32_t lo = cvt_e2m1x2(p[0] * s, p[1] * s);
+        uint32_t hi = cvt_e2m1x2(p[2] * s, p[3] * s);
+        code16 = (lo & 0xffu) | ((hi & 0xffu) << 8);
+        byte = static_cast<uint32_t>(e + 127);
+    }
+}
+
+template <int PRODUCER>
+__global__ void __launch_bounds__(kWarpsPerCta * 32)
+probgen_kernel(const float* __restrict__ scores, int64_t ld, const float* __restrict__ row_max,
+               int64_t rows, int64_t cols, ProducerConsts K, uint8_t* __restrict__ codes,
+               uint8_t* __restrict__ scales)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t segs_per_row = (cols + kSegCols - 1) / kSegCols;
+    const int64_t n_tasks = rows * segs_per_row;
+    const int64_t nblk = (cols + kMxBlock - 1) / kMxBlock;
+    const int64_t warp0 = static_cast<int64_t>(blockIdx.x) * kWarpsPerCta + (threadIdx.x >> 5);
+    const int64_t n_warps = static_cast<int64_t>(gridDim.x) * kWarpsPerCta;
+
+    for (int64_t task = warp0; task < n_tasks; task += n_warps) {
+        const int64_t row = task / segs_per_row;
+        const int64_t c0 = (task - row * segs_per_row) * kSegCols;
+        const float* src = scores + row * ld + c0;
+        const float m_s = __ldg(row_max + row);
+        uint8_t* crow = codes + row * nblk * (kMxBlock / 2) + c0 / 2;
+        uint8_t* srow = scales + row * nblk + c0 / kMxBlock;
+        const bool full = c0 + kSegCols <= cols;
+
+        float r[8][4];
+        if (full) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                float4 v = __ldcs(reinterpret_cast<const float4*>(src) + i * 32 + lane);
+                r[i][0] = v.x; r[i][1] = v.y; r[i][2] = v.z; r[i][3] = v.w;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    int64_t c = c0 + (i * 32 + lane) * 4 + u;
+                    r[i][u] = c < cols ? __ldcs(scores + row * ld + c) : -INFINITY;
+                }
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            uint32_t code16, byte;
+            produce_block<PRODUCER>(r[i], m_s, K, code16, byte);
+            const int64_t blk_col = c0 + (i * 32 + lane) / 8 * kMxBlock;   // first column of this lane's block
+            if (full || blk_col < cols) {
+                *reinterpret_cast<uint16_t*>(crow + i * 64 + lane * 2) = static_cast<uint16_t>(code16);
+                if ((lane & 7) == 0) srow[i * 4 + (lane >> 3)] = static_cast<uint8_t>(byte);
+            }
+        }
+    }
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+efq_status_t launch_probgen(int producer, const float* scores, int64_t ld, const float* row_max, int64_t rows,
+                            int64_t cols, float sigma, float tau, float h, uint8_t* codes, uint8_t* scales,
+                            cudaStream_t stream)
+{
+    if (rows < 0 || cols < 0) return EFQ_ERR_INVALID_ARG;
+    if (rows == 0 || cols == 0) return EFQ_OK;
+    if (!scores || !row_max || !codes || !scales) return EFQ_ERR_INVALID_ARG;
+    if (!isfinite(sigma) || !isfinite(tau) || !isfinite(h) || !(h > 0.0f)) return EFQ_ERR_INVALID_ARG;
+    if (ld < cols) return EFQ_ERR_INVALID_ARG;
+    if (!aligned16(scores) || (ld & 3) != 0 || !aligned16(codes)) return EFQ_ERR_ALIGNMENT;
+
+    int dev = 0, major = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return EFQ_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return EFQ_ERR_CUDA;
+    if (major != 10) return EFQ_ERR_ARCH;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return EFQ_ERR_CUDA;
+
+    ProducerConsts K = make_producer_consts(sigma, tau, h);
+    const int64_t n_tasks = rows * ((cols + kSegCols - 1) / kSegCols);
+    int64_t ctas = (n_tasks + kWarpsPerCta - 1) / kWarpsPerCta;
+    const int64_t cap = static_cast<int64_t>(sms) * 8 * 64;   // whole waves of 8 resident CTAs per SM
+    if (ctas > cap) ctas = cap;
+    dim3 grid(static_cast<unsigned>(ctas)), block(kWarpsPerCta * 32);
+    switch (producer) {
+        case kEfq:  probgen_kernel<kEfq><<<grid, block, 0, stream>>>(scores, ld, row_max, rows, cols, K, codes, scales); break;
+        case kEtq4: probgen_kernel<kEtq4><<<grid, block, 0, stream>>>(scores, ld, row_max, rows, cols, K, codes, scales); break;
+        case kEtq6: probgen_kernel<kEtq6><<<grid, block, 0, stream>>>(scores, ld, row_max, rows, cols, K, codes, scales); break;
+        default: return EFQ_ERR_INVALID_ARG;
+    }
+    return cudaGetLastError() == cudaSuccess ? EFQ_OK : EFQ_ERR_CUDA;
+}
+
+}  // namespace efq
+
+extern "C" efq_status_t efq_probgen(const float* scores, int64_t ld, const float* row_max, int64_t rows,
+                                    int64_t cols, float score_scale, const efq_params_t* params,
+                                    uint8_t* codes, uint8_t* scales, void* stream)
+{
+    float tau = -3.06f, h = 2.30f;
+    if (params) {
+        if (params->variant != 0) return EFQ_ERR_UNSUPPORTED;
+        tau = params->tau;
+        h = params->h;
+    }
+    return efq::launch_probgen(efq::kEfq, scores, ld, row_max, rows, cols, score_scale, tau, h, codes, scales,
+                               static_cast<cudaStream_t>(stream));
+}
+
+extern "C" efq_status_t exp_then_quantize_probgen(const float* scores, int64_t ld, const float* row_max,
+                                                  int64_t rows, int64_t cols, float score_scale, int scale_mode,
+                                                  uint8_t* codes, uint8_t* scales, void* stream)
+{
+    if (scale_mode != 0 && scale_mode != 1) return EFQ_ERR_INVALID_ARG;
+    return efq::launch_probgen(scale_mode == 0 ? efq::kEtq4 : efq::kEtq6, scores, ld, row_max, rows, cols,
+                               score_scale, 0.0f, 1.0f, codes, scales, static_cast<cudaStream_t>(stream));
+}
