@@ -107,7 +107,7 @@ size_t efq_attention_workspace_bytes(int B, int Hq, int Hkv, int64_t Sq, int64_t
  *   o        fp32 [B, Hq, Sq, d]
  *   causal   nonzero: query i sees keys t <= i + Sk - Sq (bottom-right aligned)
  *   softmax_scale  <= 0 selects 1/sqrt(d)
- *   workspace  device, 1024-byte aligned, >= efq_attention_workspace_bytes(...)
+ *   workspace  device, 256-byte aligned, >= efq_attention_workspace_bytes(...)
  * Q, K (blocks of 32 along d) and V (blocks of 32 along keys) are first quantised to MXFP4
  * (shared exponent floor(log2 amax) - 2, round-to-nearest-even, saturating); a query row with
  * no visible key yields zeros.  d must be 128 (UNSUPPORTED otherwise). */
@@ -123,6 +123,19 @@ efq_status_t exp_then_quantize_attention_fwd(const void* q, const void* k, const
                                              int Hq, int Hkv, int64_t Sq, int64_t Sk, int d, int causal,
                                              float softmax_scale, int scale_mode, void* workspace,
                                              size_t workspace_bytes, const efq_debug_t* debug, void* stream);
+
+/* The two halves of efq_attention_fwd as separate calls, for callers that reuse quantised operands
+ * (K/V shared by several forwards) or time the stages separately.
+ * efq_quantize_qkv: operand preparation only (bf16 -> MXFP4 into the workspace; resets the status word).
+ * efq_attention_fwd_quantized: the fused forward on a workspace prepared by efq_quantize_qkv for the
+ * same shape; producer 0 = EFQ, 1 = exp-then-quantize scale4, 2 = exp-then-quantize scale6.
+ * Arguments, layouts and errors as for efq_attention_fwd. */
+efq_status_t efq_quantize_qkv(const void* q, const void* k, const void* v, int B, int Hq, int Hkv, int64_t Sq,
+                              int64_t Sk, int d, void* workspace, size_t workspace_bytes, void* stream);
+efq_status_t efq_attention_fwd_quantized(float* o, int B, int Hq, int Hkv, int64_t Sq, int64_t Sk, int d, int causal,
+                                         float softmax_scale, int producer, const efq_params_t* params,
+                                         void* workspace, size_t workspace_bytes, const efq_debug_t* debug,
+                                         void* stream);
 
 /* End-to-end form with HOST inputs and output: copies q/k/v from (preferably pinned) host
  * memory into caller-owned device staging buffers, runs the forward selected by `producer`

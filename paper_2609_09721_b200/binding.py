@@ -21,7 +21,8 @@ STATUS_NAMES = ["EFQ_OK", "EFQ_ERR_INVALID_ARG", "EFQ_ERR_UNSUPPORTED", "EFQ_ERR
 
 # every symbol include/efq.h declares
 EXPORTS = ["efq_probgen", "exp_then_quantize_probgen", "efq_attention_workspace_bytes", "efq_attention_fwd",
-           "exp_then_quantize_attention_fwd", "efq_attention_fwd_host", "efq_poll_status",
+           "exp_then_quantize_attention_fwd", "efq_quantize_qkv", "efq_attention_fwd_quantized",
+           "efq_attention_fwd_host", "efq_poll_status",
            "efq_fp4_mma_peak_probe", "efq_status_string", "efq_version"]
 
 
@@ -65,6 +66,11 @@ def lib() -> C.CDLL:
         L.exp_then_quantize_attention_fwd.restype = i32
         L.exp_then_quantize_attention_fwd.argtypes = [vp, vp, vp, vp, i32, i32, i32, i64, i64, i32, i32, f32, i32,
                                                       vp, C.c_size_t, C.POINTER(EfqDebug), vp]
+        L.efq_quantize_qkv.restype = i32
+        L.efq_quantize_qkv.argtypes = [vp, vp, vp, i32, i32, i32, i64, i64, i32, vp, C.c_size_t, vp]
+        L.efq_attention_fwd_quantized.restype = i32
+        L.efq_attention_fwd_quantized.argtypes = [vp, i32, i32, i32, i64, i64, i32, i32, f32, i32,
+                                                  C.POINTER(EfqParams), vp, C.c_size_t, C.POINTER(EfqDebug), vp]
         L.efq_attention_fwd_host.restype = i32
         L.efq_attention_fwd_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i64, i64, i32, i32, f32,
                                              i32, C.POINTER(EfqParams), vp, C.c_size_t, vp]
@@ -208,6 +214,28 @@ def exp_then_quantize_attention_fwd(q, k, v, causal: bool = False, softmax_scale
                                                workspace.data_ptr(), workspace.numel(),
                                                C.byref(debug.c) if debug is not None else None, _stream(stream))
     _check(st, "exp_then_quantize_attention_fwd")
+    return o
+
+
+def efq_quantize_qkv(q, k, v, workspace, stream=None):
+    """Operand preparation only: bf16 Q/K/V -> MXFP4 copies in the workspace."""
+    B, Hq, Hkv, Sq, Sk, d, _, workspace = _attn_args(q, k, v, q, workspace)
+    st = lib().efq_quantize_qkv(q.data_ptr(), k.data_ptr(), v.data_ptr(), B, Hq, Hkv, Sq, Sk, d,
+                                workspace.data_ptr(), workspace.numel(), _stream(stream))
+    _check(st, "efq_quantize_qkv")
+    return workspace
+
+
+def efq_attention_fwd_quantized(o, shape, workspace, causal: bool = False, softmax_scale: float = 0.0,
+                                producer: int = 0, params=None, debug: DebugDump = None, stream=None):
+    """The fused forward on a workspace prepared by efq_quantize_qkv; shape = (B, Hq, Hkv, Sq, Sk, d)."""
+    B, Hq, Hkv, Sq, Sk, d = shape
+    p = _params(params)
+    st = lib().efq_attention_fwd_quantized(o.data_ptr(), B, Hq, Hkv, Sq, Sk, d, int(bool(causal)), float(softmax_scale),
+                                           int(producer), C.byref(p) if p is not None else None,
+                                           workspace.data_ptr(), workspace.numel(),
+                                           C.byref(debug.c) if debug is not None else None, _stream(stream))
+    _check(st, "efq_attention_fwd_quantized")
     return o
 
 

@@ -1,0 +1,720 @@
+// Fused block-scaled FP4 attention forward with in-register probability generation
+// (Algorithm 2 looped over KV tiles, Algorithm 1 per 32-key microscaling block), sm_100a.
+//
+// One CTA owns one 128-row query tile of one (batch, head) and walks the KV tiles of width 128:
+//   warp 0      TMA producer: Q tile once, then K_j / V^T_j code tiles (SW64 layout) and their
+//               512-byte scale tiles through 3-stage mbarrier rings
+//   warp 1      MMA issuer (one elected thread): scale tiles smem -> TMEM (tcgen05.cp), then
+//               S_j = Q^ K^_j^T  and  [dA | dl] = P~_j [V^_j | 1]  as kind::mxf4 block-scaled MMAs,
+//               FP32 accumulators in TMEM.  The 16 "ones" rows appended to V^T give the denominator
+//               P~1 from the very operand that feeds the numerator.
+//   warps 2-9   probability generation: thread = (query row, half of the 128 keys).  Scores come
+//               from TMEM straight into registers; block maxima and the running row maximum are
+//               thread-local plus one shared-memory exchange between the two halves; codes go as
+//               16-byte packed stores into the swizzled shared-memory A operand, scale bytes into
+//               the scale tile.  No FP16/FP32 probability tile exists anywhere.
+// The online recurrence is unchanged: when a row's maximum grows, the accumulator rows in TMEM
+// are rescaled by alpha = exp(m_old - m_new) before the next P~V MMA is released.
+//
+// TMEM columns: S double buffer 2 x 128 | O 144 (128 channels + 16 denominator) | scale factors.
+// Every wait is bounded; on expiry the CTA records EFQ_ERR_DEVICE_TIMEOUT in the workspace status
+// word, all roles drain, TMEM is released and the kernel returns.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "efq_common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace efq {
+
+cudaError_t launch_quantize_rows(const void* x, int64_t n_heads, int64_t S, int64_t S_pad, uint8_t* codes, uint8_t* sf,
+                                 cudaStream_t stream);
+cudaError_t launch_quantize_v(const void* v, int64_t n_heads, int64_t S, int64_t S_pad, uint8_t* vt_codes, uint8_t* sf,
+                              cudaStream_t stream);
+
+namespace {
+
+constexpr int kTile = 128;            // query rows per CTA and keys per KV tile (Bc)
+constexpr int kStages = 3;            // K and V ring depth
+constexpr int kThreads = 320;         // 10 warps
+constexpr int kSoftmaxWarps = 8;
+constexpr int kTileBytes = kTile * 64;          // 128 rows x 64 B of packed E2M1
+constexpr int kSfBytes = 512;
+constexpr int kVStageBytes = kTileBytes + 1024; // + 16 ones rows
+constexpr uint64_t kTimeoutCycles = 1500000000ull;
+
+// TMEM column map
+constexpr uint32_t kColS = 0;         // 2 x 128
+constexpr uint32_t kColO = 256;       // 144
+constexpr uint32_t kColSfQ = 400;     // 4
+constexpr uint32_t kColSfK = 404;     // 2 x 4
+constexpr uint32_t kColSfP = 412;     // 2 x 4
+constexpr uint32_t kColSfV = 420;     // 2 x 8 (4 for V, 4 for the ones rows)
+constexpr uint32_t kTmemCols = 512;
+
+struct __align__(1024) Smem {
+    uint8_t q[kTileBytes];
+    uint8_t k[kStages][kTileBytes];
+    uint8_t v[kStages][kVStageBytes];
+    uint8_t p[2][kTileBytes];
+    uint8_t sf_q[kSfBytes];
+    uint8_t sf_k[kStages][kSfBytes];
+    uint8_t sf_v[kStages][kSfBytes];
+    uint8_t sf_p[2][kSfBytes];
+    uint8_t sf_ones[kSfBytes];
+    float xchg[2][2][kTile];
+    uint64_t q_full;
+    uint64_t k_full[kStages], k_empty[kStages];
+    uint64_t v_full[kStages], v_empty[kStages];
+    uint64_t s_full[2], s_empty[2];
+    uint64_t p_full[2], p_empty[2];
+    uint64_t x_bar[2][4];   // row-maximum exchange between the two halves of a lane quarter
+    uint32_t tmem_base;
+    volatile uint32_t abort_flag;
+};
+
+struct FwdParams {
+    int B, Hq, Hkv;
+    int64_t Sq, Sk, Sq_pad, Sk_pad;
+    int causal;
+    int producer;             // 0 EFQ, 1 ETQ scale4, 2 ETQ scale6
+    ProducerConsts K;
+    const uint8_t* sf_q;      // [B*Hq*Sq_pad/128][512]
+    const uint8_t* sf_k;      // [B*Hkv*Sk_pad/128][512]
+    const uint8_t* sf_v;
+    float* o;
+    uint32_t* status;
+    efq_debug_t dbg;
+    int has_dbg;
+};
+
+// Warp-collective bounded wait: lane 0 polls, the verdict is broadcast.  Returns false on timeout/abort.
+__device__ __forceinline__ bool wait_barrier(uint64_t* bar, uint32_t parity, Smem* sm, uint32_t* status)
+{
+    uint32_t ok = 1;
+    if ((threadIdx.x & 31) == 0) {
+        if (!ptx::mbar_try_wait(bar, parity)) {
+            const long long t0 = clock64();
+            while (true) {
+                if (ptx::mbar_try_wait(bar, parity)) break;
+                if (sm->abort_flag) { ok = 0; break; }
+                if (static_cast<uint64_t>(clock64() - t0) > kTimeoutCycles) {
+                    ok = 0;
+                    sm->abort_flag = 1;
+                    atomicExch(status, static_cast<uint32_t>(EFQ_ERR_DEVICE_TIMEOUT));
+                    break;
+                }
+            }
+        }
+    }
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    return ok != 0;
+}
+
+__device__ __forceinline__ uint32_t p_swizzled_offset(uint32_t row, uint32_t chunk)
+{
+    return (row >> 3) * 512u + (row & 7u) * 64u + ((chunk ^ ((row >> 1) & 3u)) << 4);
+}
+
+// 32 scores of one microscaling block -> 16 bytes of codes + scale byte (EFQ: Algorithm 1).
+template <int PRODUCER>
+__device__ __forceinline__ void produce32(const float* r, float rmax, float m_s, const ProducerConsts& K, uint4& codes,
+                                          uint32_t& byte)
+{
+    uint32_t w[4];
+    if (PRODUCER == 0) {
+        BlockScale s = efq_block_scale(rmax, m_s, K);
+        byte = s.byte;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            uint32_t word = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) word |= efq_code(r[q * 8 + i], K.A, s.Bb) << (4 * i);
+            w[q] = s.live ? word : 0u;
+        }
+    } else {
+        float p[32];
+        float amax = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            float x = __fsub_rn(__fmul_rn(K.sigma, r[i]), m_s);
+            p[i] = ex2_approx(__fmul_rn(x, K.LOG2E));
+            amax = fmaxf(amax, p[i]);
+        }
+        if (amax == 0.0f) {
+            byte = 0;
+            w[0] = w[1] = w[2] = w[3] = 0;
+        } else {
+            const uint32_t bits = __float_as_uint(amax);
+            const int E = static_cast<int>((bits >> 23) & 0xffu) - 127;
+            int e = PRODUCER == 1 ? E - 2 : ((bits & 0x7fffffu) > 0x400000u ? E - 1 : E - 2);
+            e = max(e, -127);
+            const float s = __uint_as_float(static_cast<uint32_t>(127 - e) << 23);
+            byte = static_cast<uint32_t>(e + 127);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                uint32_t word = 0;
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    word |= (cvt_e2m1x2(p[q * 8 + 2 * i] * s, p[q * 8 + 2 * i + 1] * s) & 0xffu) << (8 * i);
+                w[q] = word;
+            }
+        }
+    }
+    codes = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+template <int PRODUCER, bool DEBUG>
+__global__ void __launch_bounds__(kThreads, 1)
+attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                     const __grid_constant__ CUtensorMap map_v, const FwdParams P)
+{
+    extern __shared__ uint8_t smem_raw[];
+    Smem* sm = reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    // ---- work item: heaviest query tiles first, the heads of a GQA group adjacent
+    const int64_t n_qtiles = P.Sq_pad / kTile;
+    const int64_t bh_count = static_cast<int64_t>(P.B) * P.Hq;
+    const int64_t item = blockIdx.x;
+    const int64_t qt = n_qtiles - 1 - item / bh_count;
+    const int64_t bh = item % bh_count;
+    const int b = static_cast<int>(bh / P.Hq);
+    const int hq = static_cast<int>(bh % P.Hq);
+    const int hkv = hq / (P.Hq / P.Hkv);
+    const int64_t q0 = qt * kTile;
+    const int64_t shift = P.Sk - P.Sq;                     // causal: query i sees keys <= i + shift
+    int64_t n_tiles = (P.Sk + kTile - 1) / kTile;
+    if (P.causal) {
+        int64_t last_row = q0 + kTile - 1 < P.Sq ? q0 + kTile - 1 : P.Sq - 1;
+        int64_t last_key = last_row + shift;               // may be negative: nothing visible
+        int64_t need = last_key < 0 ? 0 : last_key / kTile + 1;
+        if (need < n_tiles) n_tiles = need;
+    }
+
+    // ---- setup
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(&sm->q_full, 1);
+        for (int s = 0; s < kStages; ++s) {
+            ptx::mbar_init(&sm->k_full[s], 1);
+            ptx::mbar_init(&sm->k_empty[s], 1);
+            ptx::mbar_init(&sm->v_full[s], 1);
+            ptx::mbar_init(&sm->v_empty[s], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            ptx::mbar_init(&sm->s_full[i], 1);
+            ptx::mbar_init(&sm->s_empty[i], kSoftmaxWarps);
+            ptx::mbar_init(&sm->p_full[i], kSoftmaxWarps);
+            ptx::mbar_init(&sm->p_empty[i], 1);
+            for (int qd = 0; qd < 4; ++qd) ptx::mbar_init(&sm->x_bar[i][qd], 2);
+        }
+        sm->abort_flag = (*reinterpret_cast<volatile uint32_t*>(P.status) != 0u) ? 1u : 0u;
+        ptx::mbar_init_fence();
+    }
+    // constant parts of the B operand of P~V: 16 rows of E2M1 1.0 (0x22) after each V^T stage, unit scales
+    for (int i = threadIdx.x; i < kStages * 256; i += kThreads)
+        reinterpret_cast<uint32_t*>(sm->v[i / 256] + kTileBytes)[i % 256] = 0x22222222u;
+    for (int i = threadIdx.x; i < kSfBytes / 4; i += kThreads)
+        reinterpret_cast<uint32_t*>(sm->sf_ones)[i] = (i < 64 && (i & 3) == 0) ? 0x7f7f7f7fu : 0u;
+    ptx::fence_proxy_async_smem();
+    if (warp == 1) ptx::tmem_alloc(&sm->tmem_base, kTmemCols);
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem = sm->tmem_base;
+    const bool run = sm->abort_flag == 0 && n_tiles > 0;
+
+    if (run && warp == 0) {
+        // =============================== TMA producer ===============================
+        if (lane == 0) {
+            ptx::mbar_arrive_expect_tx(&sm->q_full, kTileBytes + kSfBytes);
+            ptx::tma_load_2d(sm->q, &map_q, 0, static_cast<int>(bh * P.Sq_pad + q0), &sm->q_full);
+            ptx::bulk_load_1d(sm->sf_q, P.sf_q + (bh * n_qtiles + qt) * kSfBytes, kSfBytes, &sm->q_full);
+        }
+        const int64_t kvh = static_cast<int64_t>(b) * P.Hkv + hkv;
+        const int64_t kv_tiles = P.Sk_pad / kTile;
+        for (int64_t j = 0; j < n_tiles; ++j) {
+            const int s = static_cast<int>(j % kStages);
+            const uint32_t ph = static_cast<uint32_t>((j / kStages) & 1);
+            if (!wait_barrier(&sm->k_empty[s], ph ^ 1u, sm, P.status)) break;
+            if (lane == 0) {
+                ptx::mbar_arrive_expect_tx(&sm->k_full[s], kTileBytes + kSfBytes);
+                ptx::tma_load_2d(sm->k[s], &map_k, 0, static_cast<int>(kvh * P.Sk_pad + j * kTile), &sm->k_full[s]);
+                ptx::bulk_load_1d(sm->sf_k[s], P.sf_k + (kvh * kv_tiles + j) * kSfBytes, kSfBytes, &sm->k_full[s]);
+            }
+            if (!wait_barrier(&sm->v_empty[s], ph ^ 1u, sm, P.status)) break;
+            if (lane == 0) {
+                ptx::mbar_arrive_expect_tx(&sm->v_full[s], kTileBytes + kSfBytes);
+                ptx::tma_load_2d(sm->v[s], &map_v, static_cast<int>(j * 64), static_cast<int>(kvh * 128), &sm->v_full[s]);
+                ptx::bulk_load_1d(sm->sf_v[s], P.sf_v + (kvh * kv_tiles + j) * kSfBytes, kSfBytes, &sm->v_full[s]);
+            }
+        }
+    } else if (run && warp == 1) {
+        // =============================== MMA issuer ===============================
+        const uint32_t q_addr = ptx::smem_u32(sm->q);
+        bool ok = wait_barrier(&sm->q_full, 0, sm, P.status);
+        ptx::tc_fence_after_sync();
+        if (ok && lane == 0) {
+            ptx::tmem_cp_sf(tmem + kColSfQ, ptx::smem_desc(ptx::smem_u32(sm->sf_q), 16, 128, ptx::kLayoutNone));
+            const uint64_t d1 = ptx::smem_desc(ptx::smem_u32(sm->sf_ones), 16, 128, ptx::kLayoutNone);
+            ptx::tmem_cp_sf(tmem + kColSfV + 4, d1);
+            ptx::tmem_cp_sf(tmem + kColSfV + 12, d1);
+        }
+        // QK_j: S[j&1] = Q K_j^T
+        auto issue_qk = [&](int64_t j) -> bool {
+            const int s = static_cast<int>(j % kStages);
+            const uint32_t ph = static_cast<uint32_t>((j / kStages) & 1);
+            const int sb = static_cast<int>(j & 1);
+            if (!wait_barrier(&sm->k_full[s], ph, sm, P.status)) return false;
+            if (!wait_barrier(&sm->s_empty[sb], static_cast<uint32_t>((j >> 1) & 1) ^ 1u, sm, P.status)) return false;
+            ptx::tc_fence_after_sync();
+            if (lane == 0) {
+                const uint32_t sfk = tmem + kColSfK + 4 * sb;
+                ptx::tmem_cp_sf(sfk, ptx::smem_desc(ptx::smem_u32(sm->sf_k[s]), 16, 128, ptx::kLayoutNone));
+                const uint32_t k_addr = ptx::smem_u32(sm->k[s]);
+#pragma unroll
+                for (uint32_t kk = 0; kk < 2; ++kk) {
+                    const uint32_t id = kk * 2;
+                    ptx::mma_mxf4(tmem + kColS + 128 * sb, ptx::smem_desc(q_addr + 32 * kk, 16, 512, ptx::kLayoutSw64),
+                                  ptx::smem_desc(k_addr + 32 * kk, 16, 512, ptx::kLayoutSw64), ptx::mxf4_idesc(128, id),
+                                  (tmem + kColSfQ) | (id << 30), sfk | (id << 30), kk);
+                }
+                ptx::mma_commit(&sm->k_empty[s]);
+                ptx::mma_commit(&sm->s_full[sb]);
+            }
+            __syncwarp();
+            return true;
+        };
+        if (ok) ok = issue_qk(0);
+        for (int64_t j = 0; ok && j < n_tiles; ++j) {
+            if (j + 1 < n_tiles) {
+                ok = issue_qk(j + 1);
+                if (!ok) break;
+            }
+            const int s = static_cast<int>(j % kStages);
+            const uint32_t ph = static_cast<uint32_t>((j / kStages) & 1);
+            const int pb = static_cast<int>(j & 1);
+            if (!wait_barrier(&sm->v_full[s], ph, sm, P.status)) { ok = false; break; }
+            if (!wait_barrier(&sm->p_full[pb], static_cast<uint32_t>((j >> 1) & 1), sm, P.status)) { ok = false; break; }
+            ptx::tc_fence_after_sync();
+            if (lane == 0) {
+                const uint32_t sfp = tmem + kColSfP + 4 * pb;
+                const uint32_t sfv = tmem + kColSfV + 8 * pb;
+                ptx::tmem_cp_sf(sfp, ptx::smem_desc(ptx::smem_u32(sm->sf_p[pb]), 16, 128, ptx::kLayoutNone));
+                ptx::tmem_cp_sf(sfv, ptx::smem_desc(ptx::smem_u32(sm->sf_v[s]), 16, 128, ptx::kLayoutNone));
+                const uint32_t p_addr = ptx::smem_u32(sm->p[pb]);
+                const uint32_t v_addr = ptx::smem_u32(sm->v[s]);
+#pragma unroll
+                for (uint32_t kk = 0; kk < 2; ++kk) {
+                    const uint32_t id = kk * 2;
+                    ptx::mma_mxf4(tmem + kColO, ptx::smem_desc(p_addr + 32 * kk, 16, 512, ptx::kLayoutSw64),
+                                  ptx::smem_desc(v_addr + 32 * kk, 16, 512, ptx::kLayoutSw64), ptx::mxf4_idesc(144, id),
+                                  sfp | (id << 30), sfv | (id << 30), (j > 0 || kk > 0) ? 1u : 0u);
+                }
+                ptx::mma_commit(&sm->v_empty[s]);
+                ptx::mma_commit(&sm->p_empty[pb]);
+            }
+            __syncwarp();
+        }
+    } else if (run && warp >= 2) {
+        // =============================== probability generation ===============================
+        const int quarter = warp & 3;                       // TMEM lane quarter this warp may touch
+        const int half = (warp - 2) >> 2;                   // which 64 keys of the tile
+        const uint32_t row = quarter * 32 + lane;           // row inside the query tile
+        const int64_t grow = q0 + row;                      // global query row
+        const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
+        const ProducerConsts K = P.K;
+        int64_t limit = P.causal ? grow + shift : P.Sk - 1; // last visible key of this row
+        if (limit > P.Sk - 1) limit = P.Sk - 1;
+        const bool dbg_row = DEBUG && P.has_dbg && b == P.dbg.batch && hq == P.dbg.head && grow >= P.dbg.q_begin &&
+                             grow < P.dbg.q_end && grow < P.Sq;
+        const int64_t drow = grow - P.dbg.q_begin;
+        const int64_t nblk_all = (P.Sk + 31) / 32;
+        const int64_t ntile_all = (P.Sk + kTile - 1) / kTile;
+
+        float m_raw = -INFINITY;
+        float m_s = -INFINITY;
+        bool ok = true;
+        for (int64_t j = 0; j < n_tiles; ++j) {
+            const int sb = static_cast<int>(j & 1);
+            const uint32_t ph2 = static_cast<uint32_t>((j >> 1) & 1);
+            if (!wait_barrier(&sm->s_full[sb], ph2, sm, P.status)) { ok = false; break; }
+            ptx::tc_fence_after_sync();
+            uint32_t sr[64];
+            const uint32_t s_addr = tmem + lane_base + kColS + 128 * sb + 64 * half;
+            ptx::tmem_ld32<0>(s_addr, sr);
+            ptx::tmem_ld32<32>(s_addr + 32, sr);
+            ptx::tmem_wait_ld();
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&sm->s_empty[sb]);
+
+            float r[64];
+            const int64_t key0 = j * kTile + 64 * half;
+            const bool need_mask = key0 + 63 > limit;
+#pragma unroll
+            for (int i = 0; i < 64; ++i) {
+                r[i] = __uint_as_float(sr[i]);
+                if (need_mask && key0 + i > limit) r[i] = -INFINITY;
+            }
+            float bmax[2];
+#pragma unroll
+            for (int g = 0; g < 2; ++g) {
+                float m = r[g * 32];
+#pragma unroll
+                for (int i = 1; i < 32; ++i) m = fmaxf(m, r[g * 32 + i]);
+                bmax[g] = m;
+            }
+            // running row maximum (Eq. rowmax-update): exchange the two halves' maxima
+            const float mine = fmaxf(bmax[0], bmax[1]);
+            sm->xchg[sb][half][row] = mine;
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&sm->x_bar[sb][quarter]);
+            if (!wait_barrier(&sm->x_bar[sb][quarter], ph2, sm, P.status)) { ok = false; break; }
+            const float other = sm->xchg[sb][half ^ 1][row];
+            const float m_new = fmaxf(m_raw, fmaxf(mine, other));
+            const float m_s_new = __fmul_rn(K.sigma, m_new);
+            const bool grew = m_new > m_raw && m_raw != -INFINITY;   // history exists and must be rescaled
+            const float alpha = grew ? ex2_approx(__fmul_rn(__fsub_rn(m_s, m_s_new), K.LOG2E)) : 1.0f;
+            m_raw = m_new;
+            m_s = m_s_new;
+
+            // P buffer sb free?  (P~V of tile j-2 finished)
+            if (!wait_barrier(&sm->p_empty[sb], ph2 ^ 1u, sm, P.status)) { ok = false; break; }
+            uint32_t bytes[2];
+#pragma unroll
+            for (int g = 0; g < 2; ++g) {
+                uint4 codes;
+                produce32<PRODUCER>(&r[g * 32], bmax[g], m_s, K, codes, bytes[g]);
+                if (m_new == -INFINITY) { codes = make_uint4(0, 0, 0, 0); bytes[g] = 0; }
+                *reinterpret_cast<uint4*>(sm->p[sb] + p_swizzled_offset(row, 2 * half + g)) = codes;
+                if (DEBUG && dbg_row) {
+                    const int64_t blk = (key0 + 32 * g) / 32;
+                    if (blk < nblk_all) {
+                        if (P.dbg.codes) *reinterpret_cast<uint4*>(P.dbg.codes + (drow * nblk_all + blk) * 16) = codes;
+                        if (P.dbg.scales) P.dbg.scales[drow * nblk_all + blk] = static_cast<uint8_t>(bytes[g]);
+                    }
+                }
+            }
+            *reinterpret_cast<uint16_t*>(sm->sf_p[sb] + (row & 31u) * 16u + (row >> 5) * 4u + 2 * half) =
+                static_cast<uint16_t>(bytes[0] | (bytes[1] << 8));
+            if (DEBUG && dbg_row) {
+                if (P.dbg.raw_scores) {
+                    for (int i = 0; i < 64; ++i)
+                        if (key0 + i < P.Sk) P.dbg.raw_scores[drow * P.Sk + key0 + i] = r[i];
+                }
+                if (P.dbg.row_max && half == 0) P.dbg.row_max[drow * ntile_all + j] = m_s;
+            }
+
+            // historical rescaling (Eq. alpha): O rows and the denominator column in TMEM
+            if (j > 0 && __any_sync(0xffffffffu, grew)) {
+                const int pv = static_cast<int>((j - 1) & 1);
+                if (!wait_barrier(&sm->p_empty[pv], static_cast<uint32_t>(((j - 1) >> 1) & 1), sm, P.status)) { ok = false; break; }
+                ptx::tc_fence_after_sync();
+                uint32_t o[64];
+                const uint32_t o_addr = tmem + lane_base + kColO + 64 * half;
+                ptx::tmem_ld32<0>(o_addr, o);
+                ptx::tmem_ld32<32>(o_addr + 32, o);
+                uint32_t lcol = 0;
+                if (half == 1) lcol = ptx::tmem_ld1(tmem + lane_base + kColO + 128);
+                ptx::tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 64; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                ptx::tmem_st32<0>(o_addr, o);
+                ptx::tmem_st32<32>(o_addr + 32, o);
+                if (half == 1) ptx::tmem_st1(tmem + lane_base + kColO + 128, __float_as_uint(__uint_as_float(lcol) * alpha));
+                ptx::tmem_wait_st();
+            }
+            ptx::fence_proxy_async_smem();
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&sm->p_full[sb]);
+        }
+        // ---- final normalisation O = A / l
+        if (ok) {
+            const int64_t jl = n_tiles - 1;
+            ok = wait_barrier(&sm->p_empty[jl & 1], static_cast<uint32_t>((jl >> 1) & 1), sm, P.status);
+        }
+        if (ok) {
+            ptx::tc_fence_after_sync();
+            uint32_t o[64];
+            const uint32_t o_addr = tmem + lane_base + kColO + 64 * half;
+            ptx::tmem_ld32<0>(o_addr, o);
+            ptx::tmem_ld32<32>(o_addr + 32, o);
+            const uint32_t lcol = ptx::tmem_ld1(tmem + lane_base + kColO + 128);
+            ptx::tmem_wait_ld();
+            if (grow < P.Sq) {
+                const float l = __uint_as_float(lcol);
+                const float inv = l > 0.0f ? 1.0f / l : 0.0f;
+                float4* dst = reinterpret_cast<float4*>(P.o + ((bh * P.Sq + grow) * 128 + 64 * half));
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    float4 v;
+                    v.x = __uint_as_float(o[4 * i + 0]) * inv;
+                    v.y = __uint_as_float(o[4 * i + 1]) * inv;
+                    v.z = __uint_as_float(o[4 * i + 2]) * inv;
+                    v.w = __uint_as_float(o[4 * i + 3]) * inv;
+                    dst[i] = v;
+                }
+            }
+        }
+    } else if (!run && warp >= 2 && sm->abort_flag == 0) {
+        // no visible key for the whole tile: rows are zero
+        const int quarter = warp & 3, half = (warp - 2) >> 2;
+        const int64_t grow = q0 + quarter * 32 + lane;
+        if (grow < P.Sq) {
+            float4* dst = reinterpret_cast<float4*>(P.o + ((bh * P.Sq + grow) * 128 + 64 * half));
+            for (int i = 0; i < 16; ++i) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    }
+
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) ptx::tmem_dealloc(tmem, kTmemCols);
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// [rows, row_bytes] u8 matrix, box 64 B x 128 rows, 64-byte swizzle
+bool encode_map(CUtensorMap* map, const void* base, uint64_t row_bytes, uint64_t rows)
+{
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {row_bytes, rows};
+    cuuint64_t strides[1] = {row_bytes};
+    cuuint32_t box[2] = {64, 128};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct Workspace {
+    size_t status, qc, qsf, kc, ksf, vt, vsf, total;
+    int64_t Sq_pad, Sk_pad;
+};
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+Workspace plan_workspace(int B, int Hq, int Hkv, int64_t Sq, int64_t Sk)
+{
+    Workspace w;
+    w.Sq_pad = (Sq + kTile - 1) / kTile * kTile;
+    w.Sk_pad = (Sk + kTile - 1) / kTile * kTile;
+    size_t off = 0;
+    w.status = off; off += 1024;
+    w.qc = off;  off = align_up(off + static_cast<size_t>(B) * Hq * w.Sq_pad * 64, 1024);
+    w.qsf = off; off = align_up(off + static_cast<size_t>(B) * Hq * (w.Sq_pad / kTile) * kSfBytes, 1024);
+    w.kc = off;  off = align_up(off + static_cast<size_t>(B) * Hkv * w.Sk_pad * 64, 1024);
+    w.ksf = off; off = align_up(off + static_cast<size_t>(B) * Hkv * (w.Sk_pad / kTile) * kSfBytes, 1024);
+    w.vt = off;  off = align_up(off + static_cast<size_t>(B) * Hkv * 128 * (w.Sk_pad / 2), 1024);
+    w.vsf = off; off = align_up(off + static_cast<size_t>(B) * Hkv * (w.Sk_pad / kTile) * kSfBytes, 1024);
+    w.total = off;
+    return w;
+}
+
+bool shape_ok(int B, int Hq, int Hkv, int64_t Sq, int64_t Sk, int d)
+{
+    return B > 0 && Hq > 0 && Hkv > 0 && Sq > 0 && Sk > 0 && d == 128 && Hq % Hkv == 0 &&
+           static_cast<int64_t>(B) * Hq * ((Sq + kTile - 1) / kTile * kTile) < (1ll << 31) &&
+           static_cast<int64_t>(B) * Hkv * ((Sk + kTile - 1) / kTile * kTile) < (1ll << 31);
+}
+
+template <int PRODUCER>
+cudaError_t launch_main(bool debug, dim3 grid, size_t smem, cudaStream_t stream, const CUtensorMap& mq, const CUtensorMap& mk,
+                        const CUtensorMap& mv, const FwdParams& P)
+{
+    cudaError_t e;
+    if (debug) {
+        e = cudaFuncSetAttribute(attention_fwd_kernel<PRODUCER, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        if (e != cudaSuccess) return e;
+        attention_fwd_kernel<PRODUCER, true><<<grid, kThreads, smem, stream>>>(mq, mk, mv, P);
+    } else {
+        e = cudaFuncSetAttribute(attention_fwd_kernel<PRODUCER, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        if (e != cudaSuccess) return e;
+        attention_fwd_kernel<PRODUCER, false><<<grid, kThreads, smem, stream>>>(mq, mk, mv, P);
+    }
+    return cudaGetLastError();
+}
+
+efq_status_t attention_impl(const void* q, const void* k, const void* v, float* o, int B, int Hq, int Hkv, int64_t Sq,
+                            int64_t Sk, int d, int causal, float softmax_scale, int producer, float tau, float h,
+                            void* workspace, size_t workspace_bytes, const efq_debug_t* debug, cudaStream_t stream,
+                            bool do_quantize, bool do_forward)
+{
+    if (!q || !k || !v || !o) return EFQ_ERR_INVALID_ARG;
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0 || Hq % Hkv != 0) return EFQ_ERR_INVALID_ARG;
+    if (d != 128) return EFQ_ERR_UNSUPPORTED;
+    if (!shape_ok(B, Hq, Hkv, Sq, Sk, d)) return EFQ_ERR_UNSUPPORTED;
+    if (!(softmax_scale > 0.0f)) softmax_scale = static_cast<float>(1.0 / sqrt(static_cast<double>(d)));
+    if (!isfinite(softmax_scale) || !isfinite(tau) || !isfinite(h) || !(h > 0.0f)) return EFQ_ERR_INVALID_ARG;
+    auto mis = [](const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0; };
+    if (mis(q, 16) || mis(k, 16) || mis(v, 16) || mis(o, 16)) return EFQ_ERR_ALIGNMENT;
+    const Workspace w = plan_workspace(B, Hq, Hkv, Sq, Sk);
+    if (!workspace || workspace_bytes < w.total) return EFQ_ERR_WORKSPACE;
+    if (mis(workspace, 256)) return EFQ_ERR_ALIGNMENT;
+
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return EFQ_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return EFQ_ERR_CUDA;
+    if (major != 10) return EFQ_ERR_ARCH;
+
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    if (do_quantize) {
+        if (cudaMemsetAsync(ws + w.status, 0, 1024, stream) != cudaSuccess) return EFQ_ERR_CUDA;
+        if (launch_quantize_rows(q, static_cast<int64_t>(B) * Hq, Sq, w.Sq_pad, ws + w.qc, ws + w.qsf, stream) != cudaSuccess) return EFQ_ERR_CUDA;
+        if (launch_quantize_rows(k, static_cast<int64_t>(B) * Hkv, Sk, w.Sk_pad, ws + w.kc, ws + w.ksf, stream) != cudaSuccess) return EFQ_ERR_CUDA;
+        if (launch_quantize_v(v, static_cast<int64_t>(B) * Hkv, Sk, w.Sk_pad, ws + w.vt, ws + w.vsf, stream) != cudaSuccess) return EFQ_ERR_CUDA;
+    }
+    if (!do_forward) return EFQ_OK;
+
+    CUtensorMap mq, mk, mv;
+    if (!encode_map(&mq, ws + w.qc, 64, static_cast<uint64_t>(B) * Hq * w.Sq_pad)) return EFQ_ERR_CUDA;
+    if (!encode_map(&mk, ws + w.kc, 64, static_cast<uint64_t>(B) * Hkv * w.Sk_pad)) return EFQ_ERR_CUDA;
+    if (!encode_map(&mv, ws + w.vt, static_cast<uint64_t>(w.Sk_pad / 2), static_cast<uint64_t>(B) * Hkv * 128)) return EFQ_ERR_CUDA;
+
+    FwdParams P;
+    P.B = B; P.Hq = Hq; P.Hkv = Hkv; P.Sq = Sq; P.Sk = Sk; P.Sq_pad = w.Sq_pad; P.Sk_pad = w.Sk_pad;
+    P.causal = causal ? 1 : 0;
+    P.producer = producer;
+    P.K = make_producer_consts(softmax_scale, tau, h);
+    P.sf_q = ws + w.qsf; P.sf_k = ws + w.ksf; P.sf_v = ws + w.vsf;
+    P.o = o;
+    P.status = reinterpret_cast<uint32_t*>(ws + w.status);
+    P.has_dbg = debug ? 1 : 0;
+    if (debug) P.dbg = *debug; else P.dbg = efq_debug_t{};
+
+    const int64_t items = (w.Sq_pad / kTile) * B * Hq;
+    dim3 grid(static_cast<unsigned>(items));
+    // more than half of the SM's shared memory: one CTA per SM, since each CTA takes all 512 TMEM columns
+    const size_t smem = sizeof(Smem) + 1024 > 120 * 1024 ? sizeof(Smem) + 1024 : 120 * 1024;
+    cudaError_t e;
+    switch (producer) {
+        case 0: e = launch_main<0>(debug != nullptr, grid, smem, stream, mq, mk, mv, P); break;
+        case 1: e = launch_main<1>(debug != nullptr, grid, smem, stream, mq, mk, mv, P); break;
+        case 2: e = launch_main<2>(debug != nullptr, grid, smem, stream, mq, mk, mv, P); break;
+        default: return EFQ_ERR_INVALID_ARG;
+    }
+    return e == cudaSuccess ? EFQ_OK : EFQ_ERR_CUDA;
+}
+
+}  // namespace
+}  // namespace efq
+
+extern "C" size_t efq_attention_workspace_bytes(int B, int Hq, int Hkv, int64_t Sq, int64_t Sk, int d)
+{
+    if (!efq::shape_ok(B, Hq, Hkv, Sq, Sk, d)) return 0;
+    return efq::plan_workspace(B, Hq, Hkv, Sq, Sk).total;
+}
+
+static bool read_params(const efq_params_t* params, float& tau, float& h, efq_status_t& st)
+{
+    tau = -3.06f;
+    h = 2.30f;
+    st = EFQ_OK;
+    if (params) {
+        if (params->variant != 0) { st = EFQ_ERR_UNSUPPORTED; return false; }
+        if (params->kv_tile != 0 && params->kv_tile != 128) { st = EFQ_ERR_UNSUPPORTED; return false; }
+        tau = params->tau;
+        h = params->h;
+    }
+    return true;
+}
+
+extern "C" efq_status_t efq_attention_fwd(const void* q, const void* k, const void* v, float* o, int B, int Hq, int Hkv,
+                                          int64_t Sq, int64_t Sk, int d, int causal, float softmax_scale,
+                                          const efq_params_t* params, void* workspace, size_t workspace_bytes,
+                                          const efq_debug_t* debug, void* stream)
+{
+    float tau, h;
+    efq_status_t st;
+    if (!read_params(params, tau, h, st)) return st;
+    return efq::attention_impl(q, k, v, o, B, Hq, Hkv, Sq, Sk, d, causal, softmax_scale, 0, tau, h, workspace,
+                               workspace_bytes, debug, static_cast<cudaStream_t>(stream), true, true);
+}
+
+extern "C" efq_status_t exp_then_quantize_attention_fwd(const void* q, const void* k, const void* v, float* o, int B,
+                                                        int Hq, int Hkv, int64_t Sq, int64_t Sk, int d, int causal,
+                                                        float softmax_scale, int scale_mode, void* workspace,
+                                                        size_t workspace_bytes, const efq_debug_t* debug, void* stream)
+{
+    if (scale_mode != 0 && scale_mode != 1) return EFQ_ERR_INVALID_ARG;
+    return efq::attention_impl(q, k, v, o, B, Hq, Hkv, Sq, Sk, d, causal, softmax_scale, 1 + scale_mode, 0.0f, 1.0f,
+                               workspace, workspace_bytes, debug, static_cast<cudaStream_t>(stream), true, true);
+}
+
+extern "C" efq_status_t efq_quantize_qkv(const void* q, const void* k, const void* v, int B, int Hq, int Hkv, int64_t Sq,
+                                         int64_t Sk, int d, void* workspace, size_t workspace_bytes, void* stream)
+{
+    const void* nz_o = reinterpret_cast<const void*>(16);   // no output is written by the preparation step
+    return efq::attention_impl(q, k, v, static_cast<float*>(const_cast<void*>(nz_o)), B, Hq, Hkv, Sq, Sk, d, 0, 0.0f, 0,
+                               -3.06f, 2.30f, workspace, workspace_bytes, nullptr, static_cast<cudaStream_t>(stream), true,
+                               false);
+}
+
+extern "C" efq_status_t efq_attention_fwd_quantized(float* o, int B, int Hq, int Hkv, int64_t Sq, int64_t Sk, int d,
+                                                    int causal, float softmax_scale, int producer,
+                                                    const efq_params_t* params, void* workspace, size_t workspace_bytes,
+                                                    const efq_debug_t* debug, void* stream)
+{
+    float tau, h;
+    efq_status_t st;
+    if (!read_params(params, tau, h, st)) return st;
+    const void* nz = reinterpret_cast<const void*>(16);   // operands already live in the workspace
+    return efq::attention_impl(nz, nz, nz, o, B, Hq, Hkv, Sq, Sk, d, causal, softmax_scale, producer, tau, h, workspace,
+                               workspace_bytes, debug, static_cast<cudaStream_t>(stream), false, true);
+}
+
+extern "C" efq_status_t efq_attention_fwd_host(const void* q_host, const void* k_host, const void* v_host, float* o_host,
+                                               void* q_dev, void* k_dev, void* v_dev, float* o_dev, int B, int Hq, int Hkv,
+                                               int64_t Sq, int64_t Sk, int d, int causal, float softmax_scale, int producer,
+                                               const efq_params_t* params, void* workspace, size_t workspace_bytes,
+                                               void* stream)
+{
+    if (!q_host || !k_host || !v_host || !o_host || !q_dev || !k_dev || !v_dev || !o_dev) return EFQ_ERR_INVALID_ARG;
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0) return EFQ_ERR_INVALID_ARG;
+    float tau, h;
+    efq_status_t st;
+    if (!read_params(params, tau, h, st)) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t qb = static_cast<size_t>(B) * Hq * Sq * d * 2, kb = static_cast<size_t>(B) * Hkv * Sk * d * 2;
+    if (cudaMemcpyAsync(q_dev, q_host, qb, cudaMemcpyHostToDevice, s) != cudaSuccess) return EFQ_ERR_CUDA;
+    if (cudaMemcpyAsync(k_dev, k_host, kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return EFQ_ERR_CUDA;
+    if (cudaMemcpyAsync(v_dev, v_host, kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return EFQ_ERR_CUDA;
+    st = efq::attention_impl(q_dev, k_dev, v_dev, o_dev, B, Hq, Hkv, Sq, Sk, d, causal, softmax_scale, producer, tau, h,
+                             workspace, workspace_bytes, nullptr, s, true, true);
+    if (st != EFQ_OK) return st;
+    if (cudaMemcpyAsync(o_host, o_dev, static_cast<size_t>(B) * Hq * Sq * d * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return EFQ_ERR_CUDA;
+    return EFQ_OK;
+}
+
+extern "C" efq_status_t efq_poll_status(void* workspace, void* stream)
+{
+    if (!workspace) return EFQ_ERR_INVALID_ARG;
+    uint32_t word = 0;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(&word, workspace, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return EFQ_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return EFQ_ERR_CUDA;
+    return word == 0 ? EFQ_OK : (word == EFQ_ERR_DEVICE_TIMEOUT ? EFQ_ERR_DEVICE_TIMEOUT : EFQ_ERR_CUDA);
+}

@@ -1,0 +1,135 @@
+// Operand preparation for the fused forward: bf16 Q, K, V -> MXFP4 (packed E2M1 codes + one E8M0
+// byte per 32 elements) in the layouts the TMA loads and tcgen05 block-scaled MMAs consume.
+// This is the surrounding kernel's "existing low-bit path" (Sec. 3.1); EFQ itself does not touch it.
+//
+// OCP microscaling rule per 32-element block: shared exponent e = floor(log2 amax) - 2 (clamped to
+// the E8M0 range), elements rounded to nearest-even E2M1 of x * 2^-e, saturating at +-6; an all-zero
+// block gets byte 0 and zero codes.
+//
+// Layouts written (S_pad = S rounded up to 128; padding rows/keys are zero codes, byte 0):
+//   Q, K codes   [B*H, S_pad, 64 B]          row-major, 2 codes per byte, element 2u in the low nibble
+//   V^T codes    [B*Hkv, 128 (channel), S_pad/2 B]   keys contiguous: the P~V contraction runs over keys
+//   scale tiles  one 512-byte tile per 128 rows (Q, K: rows = tokens, 4 blocks along d;
+//                V: rows = channels, 4 key blocks of the 128-key tile); byte of (row r, block b) at
+//                (r % 32) * 16 + (r / 32) * 4 + b, the order the scale-factor copy into TMEM expects.
+#include <cuda_bf16.h>
+
+#include "efq_common.cuh"
+
+namespace efq {
+
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t b) { return __uint_as_float(b << 16); }
+
+// 32 bf16 values (as 16 packed 32-bit words, element 2u in the low half) -> 16 bytes of codes + scale byte
+__device__ __forceinline__ void mxfp4_block(const uint32_t (&w)[16], uint4& codes, uint32_t& byte)
+{
+    uint32_t amax = 0;   // bf16 magnitudes compare like unsigned integers
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        amax = max(amax, w[i] & 0x7fffu);
+        amax = max(amax, (w[i] >> 16) & 0x7fffu);
+    }
+    if (amax == 0) {
+        codes = make_uint4(0, 0, 0, 0);
+        byte = 0;
+        return;
+    }
+    int e = static_cast<int>(amax >> 7) - 127 - 2;   // exponent field of the largest magnitude, minus 2
+    e = max(e, -127);
+    const float s = __uint_as_float(static_cast<uint32_t>(127 - e) << 23);   // 2^-e, field in [2, 254]
+    uint32_t out[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        uint32_t word = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            uint32_t v = w[q * 4 + i];
+            float lo = bf16_bits_to_float(v & 0xffffu) * s;
+            float hi = bf16_bits_to_float(v >> 16) * s;
+            word |= (cvt_e2m1x2(lo, hi) & 0xffu) << (8 * i);
+        }
+        out[q] = word;
+    }
+    codes = make_uint4(out[0], out[1], out[2], out[3]);
+    byte = static_cast<uint32_t>(e + 127);
+}
+
+__device__ __forceinline__ uint32_t sf_tile_offset(uint32_t r, uint32_t b) { return (r & 31u) * 16u + (r >> 5) * 4u + b; }
+
+// One thread per (row, 32-wide block along d); d = 128.
+__global__ void __launch_bounds__(256)
+quantize_rows_kernel(const __nv_bfloat16* __restrict__ x, int64_t n_heads, int64_t S, int64_t S_pad,
+                     uint8_t* __restrict__ codes, uint8_t* __restrict__ sf)
+{
+    const int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const int64_t total = n_heads * S_pad * 4;
+    if (t >= total) return;
+    const int blk = static_cast<int>(t & 3);
+    const int64_t prow = t >> 2;               // padded row index over all heads
+    const int64_t head = prow / S_pad;
+    const int64_t row = prow - head * S_pad;
+    uint4 c = make_uint4(0, 0, 0, 0);
+    uint32_t byte = 0;
+    if (row < S) {
+        const uint4* src = reinterpret_cast<const uint4*>(x + (head * S + row) * 128 + blk * 32);
+        uint32_t w[16];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            uint4 v = __ldg(src + i);
+            w[4 * i + 0] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
+        }
+        mxfp4_block(w, c, byte);
+    }
+    *reinterpret_cast<uint4*>(codes + prow * 64 + blk * 16) = c;
+    const int64_t tile = prow >> 7;            // S_pad is a multiple of 128, so tiles never straddle heads
+    sf[tile * 512 + sf_tile_offset(static_cast<uint32_t>(prow & 127), blk)] = static_cast<uint8_t>(byte);
+}
+
+// One thread per (32-key block, channel); consecutive threads take consecutive channels.
+__global__ void __launch_bounds__(128)
+quantize_v_kernel(const __nv_bfloat16* __restrict__ v, int64_t n_heads, int64_t S, int64_t S_pad,
+                  uint8_t* __restrict__ vt_codes, uint8_t* __restrict__ sf)
+{
+    const int ch = threadIdx.x;                               // 0..127
+    const int64_t kb = blockIdx.x;                            // key block over all heads
+    const int64_t blocks_per_head = S_pad / 32;
+    const int64_t head = kb / blocks_per_head;
+    const int64_t kblk = kb - head * blocks_per_head;
+    const uint16_t* src = reinterpret_cast<const uint16_t*>(v) + (head * S + kblk * 32) * 128 + ch;
+    uint32_t w[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const int64_t k0 = kblk * 32 + 2 * i;
+        uint32_t lo = k0 < S ? __ldg(src + (2 * i) * 128) : 0u;
+        uint32_t hi = k0 + 1 < S ? __ldg(src + (2 * i + 1) * 128) : 0u;
+        w[i] = lo | (hi << 16);
+    }
+    uint4 c;
+    uint32_t byte;
+    mxfp4_block(w, c, byte);
+    *reinterpret_cast<uint4*>(vt_codes + (head * 128 + ch) * (S_pad / 2) + kblk * 16) = c;
+    const int64_t tile = head * (S_pad / 128) + (kblk >> 2);
+    sf[tile * 512 + sf_tile_offset(static_cast<uint32_t>(ch), static_cast<uint32_t>(kblk & 3))] = static_cast<uint8_t>(byte);
+}
+
+cudaError_t launch_quantize_rows(const void* x, int64_t n_heads, int64_t S, int64_t S_pad, uint8_t* codes, uint8_t* sf,
+                                 cudaStream_t stream)
+{
+    const int64_t total = n_heads * S_pad * 4;
+    if (total == 0) return cudaSuccess;
+    quantize_rows_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, stream>>>(
+        static_cast<const __nv_bfloat16*>(x), n_heads, S, S_pad, codes, sf);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_quantize_v(const void* v, int64_t n_heads, int64_t S, int64_t S_pad, uint8_t* vt_codes, uint8_t* sf,
+                              cudaStream_t stream)
+{
+    const int64_t blocks = n_heads * (S_pad / 32);
+    if (blocks == 0) return cudaSuccess;
+    quantize_v_kernel<<<static_cast<unsigned>(blocks), 128, 0, stream>>>(static_cast<const __nv_bfloat16*>(v), n_heads, S,
+                                                                         S_pad, vt_codes, sf);
+    return cudaGetLastError();
+}
+
+}  // namespace efq

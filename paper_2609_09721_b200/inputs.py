@@ -17,6 +17,7 @@ independently and in any chunking.
 from __future__ import annotations
 
 import math
+import os
 from dataclasses import dataclass
 
 import numpy as np
@@ -53,14 +54,26 @@ def uniform(seed: int, tid: int, start: int, count: int, lane: int = 0) -> np.nd
     return ((h >> _U64(11)).astype(np.float64) + 0.5) * (1.0 / 9007199254740992.0)
 
 
+def _normal_chunk(args):
+    seed, tid, start, n, out = args
+    u1 = uniform(seed, tid, start, n, 0)
+    u2 = uniform(seed, tid, start, n, 1)
+    np.multiply(np.sqrt(-2.0 * np.log(u1)), np.cos((2.0 * math.pi) * u2), out=out)
+
+
 def normal(seed: int, tid: int, count: int, start: int = 0) -> np.ndarray:
-    """float64 N(0,1) samples for flat indices ``start .. start+count-1``."""
+    """float64 N(0,1) samples for flat indices ``start .. start+count-1`` (chunks run on a thread pool;
+    the values do not depend on the chunking)."""
     out = np.empty(count, dtype=np.float64)
-    for lo in range(0, count, _CHUNK):
-        n = min(_CHUNK, count - lo)
-        u1 = uniform(seed, tid, start + lo, n, 0)
-        u2 = uniform(seed, tid, start + lo, n, 1)
-        out[lo:lo + n] = np.sqrt(-2.0 * np.log(u1)) * np.cos((2.0 * math.pi) * u2)
+    jobs = [(seed, tid, start + lo, min(_CHUNK, count - lo), out[lo:lo + min(_CHUNK, count - lo)])
+            for lo in range(0, count, _CHUNK)]
+    if len(jobs) <= 1:
+        for j in jobs:
+            _normal_chunk(j)
+    else:
+        from concurrent.futures import ThreadPoolExecutor
+        with ThreadPoolExecutor(max_workers=min(len(jobs), os.cpu_count() or 1, 32)) as ex:
+            list(ex.map(_normal_chunk, jobs))
     return out
 
 

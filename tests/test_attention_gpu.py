@@ -1,0 +1,191 @@
+"""GPU parity of the fused FP4 attention forward against the CPU oracle, through the C ABI.
+
+Levels: (L1) the kernel's probability operand (codes + E8M0 bytes) is bit-exact given the kernel's
+own FP32 raw scores and running maxima; the raw scores themselves equal the oracle's exact dot
+products of the dequantised operands; (L2) max |O_gpu - O_oracle| <= 2e-3 end to end from the same
+bf16 inputs.  The error against exact (unquantised, FP32-softmax) attention is reported, not bounded
+tightly: the paper prints no figure for it."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_09721_b200 import binding, inputs
+
+pytestmark = pytest.mark.gpu
+
+TOL_O = 2e-3
+MEAN = (-3.06, 2.30)
+
+
+def _to_dev(bits):
+    return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def _case_tensors(case):
+    qb, kb, vb = inputs.make_qkv(case)
+    host = tuple(inputs.bf16_bits_to_f32(t) for t in (qb, kb, vb))
+    dev = tuple(_to_dev(t) for t in (qb, kb, vb))
+    return host, dev
+
+
+def _all_rows(case, head, lo, hi):
+    return np.array([(0, head, i) for i in range(lo, hi)], np.int64)
+
+
+def _visible(case, i):
+    return min(case.Sk, i + case.Sk - case.Sq + 1) if case.causal else case.Sk
+
+
+def _check_dump(oracle, case, dump, rows, params, producer="efq", want=None):
+    """L1: operand bit-exact on the kernel's own scores; raw scores equal to the oracle's."""
+    raw = dump.raw_scores.cpu().numpy()
+    codes = dump.codes.cpu().numpy()
+    scales = dump.scales.cpu().numpy()
+    ms = dump.row_max.cpu().numpy()
+    for n, (_, _, i) in enumerate(rows):
+        nv = _visible(case, int(i))
+        assert np.all(np.isfinite(raw[n, :nv])), "visible scores must be written"
+        raw[n, nv:] = -np.inf
+    oc, osc, oms = oracle.online_codes(raw, 128, case.softmax_scale, *params, producer=producer)
+    for n, (_, _, i) in enumerate(rows):
+        nt = (_visible(case, int(i)) + 127) // 128
+        assert np.array_equal(ms[n, :nt], oms[n, :nt])
+    if producer == "efq":
+        assert np.array_equal(scales, osc)
+        assert np.array_equal(codes, oc)
+    else:
+        sd = scales != osc
+        assert sd.mean() < 2e-3
+        a = oracle.unpack_codes(codes).astype(int)
+        b = oracle.unpack_codes(oc).astype(int)
+        okm = np.repeat(~sd, 32, axis=1)
+        d = np.abs(a - b)[okm]
+        assert d.max() <= 1 and (d != 0).mean() < 2e-3
+    if want is not None:
+        wraw = want["raw"]
+        fin = np.isfinite(wraw)
+        mism = (raw[fin] != wraw[fin]).mean()
+        return mism
+    return 0.0
+
+
+@pytest.mark.parametrize("params", [MEAN, (-2.90, 2.00), (-2.10, 2.70)])
+def test_single_head_1024_full_dump(oracle, params):
+    """Config: B=1, H=1, S=1024, d=128, non-causal, N(0,1) bf16."""
+    case = inputs.case_single_head(1024, seed=1)
+    (q, k, v), (dq, dk, dv) = _case_tensors(case)
+    dump = binding.DebugDump(0, 0, 0, 1024, 1024)
+    o = binding.efq_attention_fwd(dq, dk, dv, False, 0.0, params, debug=dump)
+    torch.cuda.synchronize()
+    ws_ok = o is not None
+    assert ws_ok
+    rows = _all_rows(case, 0, 0, 1024)
+    want_o, want = oracle.attention_rows(q, k, v, rows, False, case.softmax_scale, "efq", *params, dumps=True)
+    mism = _check_dump(oracle, case, dump, rows, params, want=want)
+    assert mism == 0.0, f"raw scores differ from exact dot products on a fraction {mism}"
+    assert np.array_equal(dump.codes.cpu().numpy(), want["codes"])
+    assert np.array_equal(dump.scales.cpu().numpy(), want["scales"])
+    got = o.cpu().numpy()[0, 0]
+    assert np.abs(got - want_o).max() <= TOL_O
+    exact = oracle.attention_rows(q, k, v, rows, False, case.softmax_scale, "exact")
+    print("single_head_1024: max|O_gpu-O_oracle| =", np.abs(got - want_o).max(),
+          " rel-Frobenius vs exact =", np.linalg.norm(got - exact) / np.linalg.norm(exact))
+
+
+@pytest.mark.parametrize("S,Hq,Hkv,causal,recipe", [
+    (384, 4, 2, True, "iid"), (300, 2, 1, False, "iid"), (300, 2, 2, True, "k_outliers"),
+    (1000, 4, 1, True, "lowrank"), (130, 1, 1, True, "iid"), (24, 1, 1, False, "iid"), (1, 2, 1, True, "iid"),
+])
+def test_small_shapes_efq(oracle, S, Hq, Hkv, causal, recipe):
+    case = inputs.AttentionCase("t", 1, Hq, Hkv, S, S, 128, causal, 40 + S, recipe)
+    (q, k, v), (dq, dk, dv) = _case_tensors(case)
+    head = Hq - 1
+    dump = binding.DebugDump(0, head, 0, S, S)
+    o = binding.efq_attention_fwd(dq, dk, dv, causal, 0.0, None, debug=dump)
+    torch.cuda.synchronize()
+    rows = np.array([(0, h, i) for h in range(Hq) for i in range(S)], np.int64)
+    want_o = oracle.attention_rows(q, k, v, rows, causal, case.softmax_scale, "efq")
+    got = o.cpu().numpy().reshape(-1, 128)
+    assert np.abs(got - want_o).max() <= TOL_O
+    _check_dump(oracle, case, dump, _all_rows(case, head, 0, S), MEAN)
+
+
+@pytest.mark.parametrize("Sq,Sk,causal", [(128, 512, True), (100, 700, False), (260, 200, True), (64, 4096 + 88, True)])
+def test_cross_shapes_sq_ne_sk(oracle, Sq, Sk, causal):
+    case = inputs.AttentionCase("x", 1, 2, 1, Sq, Sk, 128, causal, 77, "iid")
+    (q, k, v), (dq, dk, dv) = _case_tensors(case)
+    o = binding.efq_attention_fwd(dq, dk, dv, causal)
+    torch.cuda.synchronize()
+    rows = np.array([(0, h, i) for h in range(2) for i in range(Sq)], np.int64)
+    want_o = oracle.attention_rows(q, k, v, rows, causal, case.softmax_scale, "efq")
+    got = o.cpu().numpy().reshape(-1, 128)
+    assert np.abs(got - want_o).max() <= TOL_O
+    if causal and Sq > Sk:     # rows with no visible key are zero
+        assert np.all(got.reshape(2, Sq, 128)[:, : Sq - Sk] == 0.0)
+
+
+@pytest.mark.parametrize("mode,path", [(0, "etq"), (1, "etq6")])
+def test_exp_then_quantize_path(oracle, mode, path):
+    case = inputs.AttentionCase("t", 1, 4, 2, 640, 640, 128, True, 9, "k_outliers")
+    (q, k, v), (dq, dk, dv) = _case_tensors(case)
+    dump = binding.DebugDump(0, 1, 0, 640, 640)
+    o = binding.exp_then_quantize_attention_fwd(dq, dk, dv, True, 0.0, mode, debug=dump)
+    torch.cuda.synchronize()
+    rows = np.array([(0, h, i) for h in range(4) for i in range(640)], np.int64)
+    want_o = oracle.attention_rows(q, k, v, rows, True, case.softmax_scale, path)
+    got = o.cpu().numpy().reshape(-1, 128)
+    assert np.abs(got - want_o).max() <= 5e-3      # device exp is approximate: codes flip at knife-edges
+    _check_dump(oracle, case, dump, _all_rows(case, 1, 0, 640), MEAN, producer=path)
+    exact = oracle.attention_rows(q, k, v, rows, True, case.softmax_scale, "exact")
+    print(path, "rel-Frobenius vs exact =", np.linalg.norm(got - exact) / np.linalg.norm(exact))
+
+
+def _sampled_parity(oracle, case, n_random, label):
+    (q, k, v), (dq, dk, dv) = _case_tensors(case)
+    o = binding.efq_attention_fwd(dq, dk, dv, case.causal)
+    torch.cuda.synchronize()
+    rows = inputs.sample_rows(case, n_random)
+    want = oracle.attention_rows(q, k, v, rows, case.causal, case.softmax_scale, "efq")
+    oc = o.cpu().numpy()
+    got = oc[rows[:, 0], rows[:, 1], rows[:, 2]]
+    err = np.abs(got - want).max()
+    exact = oracle.attention_rows(q, k, v, rows[:64], case.causal, case.softmax_scale, "exact")
+    print(label, "rows", len(rows), "max|O_gpu-O_oracle| =", err, " rel-Frobenius vs exact =",
+          np.linalg.norm(got[:64] - exact) / np.linalg.norm(exact))
+    assert err <= TOL_O
+    assert np.all(np.isfinite(oc))
+
+
+def test_qwen3_shape_reduced(oracle):
+    _sampled_parity(oracle, inputs.case_qwen3_8b(2048, seed=3, Hq=8, Hkv=2), 200, "qwen3-like S=2048")
+
+
+def test_wan_shape_reduced_ragged_tail(oracle):
+    """S = 4088 = 127*32 + 24: ragged final microscaling block, non-causal, low-rank structure."""
+    _sampled_parity(oracle, inputs.case_wan22(4088, seed=5, H=3), 200, "wan-like S=4088")
+
+
+def test_qwen3_8b_16k_full_size_sampled_rows(oracle):
+    """The benchmarked configuration at full size (32 q heads / 8 kv heads, S=16384, causal)."""
+    _sampled_parity(oracle, inputs.case_qwen3_8b(16384, seed=3), 256, "qwen3-8b S=16384")
+
+
+def test_attention_argument_errors():
+    q = torch.zeros((1, 3, 128, 128), dtype=torch.bfloat16, device="cuda")
+    k = torch.zeros((1, 2, 128, 128), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(binding.EfqError) as e:
+        binding.efq_attention_fwd(q, k, k)                   # Hq % Hkv != 0
+    assert e.value.status == 1
+    q64 = torch.zeros((1, 2, 128, 64), dtype=torch.bfloat16, device="cuda")
+    assert binding.efq_attention_workspace_bytes(1, 2, 2, 128, 128, 64) == 0
+    with pytest.raises(binding.EfqError) as e:
+        binding.efq_attention_fwd(q64, q64, q64)             # d != 128
+    assert e.value.status == 2
+    q2 = torch.zeros((1, 2, 128, 128), dtype=torch.bfloat16, device="cuda")
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(binding.EfqError) as e:
+        binding.efq_attention_fwd(q2, k, k, workspace=small)
+    assert e.value.status == 4
+    ws = torch.empty(binding.efq_attention_workspace_bytes(1, 2, 2, 128, 128, 128), dtype=torch.uint8, device="cuda")
+    binding.efq_attention_fwd(q2, k, k, workspace=ws)
+    assert binding.efq_poll_status(ws) == 0
