@@ -1,0 +1,377 @@
+#!/usr/bin/env python
+"""Benchmark of the EFQ-Softmax hot path on B200.
+
+One "step" is one pass of the whole hot path over one batch of synthetic input: operand
+preparation (bf16 -> MXFP4), then the fused FP4 attention forward with EFQ probability
+generation.  Default workload: Qwen3-8B-shaped prefill attention (B=1, 32 query heads,
+8 KV heads, d=128, S=16384, causal); metric: attention forward TFLOP/s
+(4*B*Hq*Sq*Sk*d, halved for causal).
+
+    python bench.py --gpus N --steps K --warmup W            # CUDA path (rank per GPU under torchrun)
+    python bench.py --impl reference --steps K --warmup W    # the CPU oracle, bounded sample per step
+
+Prints one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2609_09721_b200 import inputs  # noqa: E402
+
+METRIC = "efq_fp4_attention_fwd_tflops"
+UNIT = "TFLOP/s"
+NOMINAL_FP4_OVER_BF16 = 4.0          # dense FP4 : dense bf16 tensor throughput on B200 (9 : 2.25 PFLOP/s)
+FALLBACK_BF16_TFLOPS = 1590.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def workload_case(name: str) -> inputs.AttentionCase:
+    if name == "qwen3_8b_16k":
+        return inputs.case_qwen3_8b(16384, seed=3)
+    if name == "qwen3_8b_128k":
+        return inputs.case_qwen3_8b(131072, seed=4)
+    if name == "wan22_32760":
+        return inputs.case_wan22(32760, seed=5)
+    if name == "single_head_1024":
+        return inputs.case_single_head(1024, seed=1)
+    if name == "qwen3_8b_2k":   # small case for smoke runs and profiler captures
+        return inputs.case_qwen3_8b(2048, seed=3)
+    raise SystemExit(f"unknown workload {name}")
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"bf16_burst": float(p["bf16_tflops"]), "bf16_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "hbm_gbs": float(p["hbm_gbs"]), "source": "measured"}
+    return {"bf16_burst": FALLBACK_BF16_TFLOPS, "bf16_sustained": 1400.0, "hbm_gbs": FALLBACK_HBM_GBS, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.lines = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.gpu), "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for ln in self.proc.stdout:
+            self.lines.append((time.time(), ln.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ts, ln in self.lines:
+            if ts < t0 - 0.05 or ts > t1 + 0.05:
+                continue
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+                power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples inside the timed region"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(smax), "reasons": sorted(reasons),
+                "power_w_max": max(power), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands, on a bounded sample of query rows per step
+# ------------------------------------------------------------------------------------------
+
+def oracle_sample_rows(case, n_rows, step):
+    u = inputs.hash_u64(1234 + step, 9, 0, 2 * n_rows)
+    rows = [(0, int(u[2 * i] % np.uint64(case.Hq)), int(u[2 * i + 1] % np.uint64(case.Sq))) for i in range(n_rows)]
+    return np.asarray(rows, dtype=np.int64)
+
+
+def rows_flops(case, rows):
+    vis = rows[:, 2] + (case.Sk - case.Sq) + 1 if case.causal else np.full(len(rows), case.Sk)
+    return float(4.0 * case.d * np.clip(vis, 0, case.Sk).sum())
+
+
+def time_oracle(case, q, k, v, n_rows, steps, warmup):
+    from oracle import efq_oracle
+    times, flops = [], []
+    for s in range(warmup + steps):
+        rows = oracle_sample_rows(case, n_rows, s)
+        t0 = time.perf_counter()
+        efq_oracle.attention_rows(q, k, v, rows, case.causal, case.softmax_scale, "efq")
+        dt = time.perf_counter() - t0
+        if s >= warmup:
+            times.append(dt)
+            flops.append(rows_flops(case, rows))
+    return sum(flops) / sum(times) / 1e12, sum(times) / len(times), efq_oracle.threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    case = workload_case(args.workload)
+    qb, kb, vb = inputs.make_qkv(case)
+    q, k, v = (inputs.bf16_bits_to_f32(t) for t in (qb, kb, vb))
+    n_rows = args.oracle_rows
+    value, sec_per_step, cores = time_oracle(case, q, k, v, n_rows, args.steps, args.warmup)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec_per_step * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": case.name, "B": case.B, "Hq": case.Hq, "Hkv": case.Hkv, "S": case.Sq, "d": case.d,
+                   "causal": case.causal, "kv_tile": 128},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"{n_rows} seeded query rows per step (all heads), EFQ path, flops = 4*d*visible keys"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------
+# CUDA arm
+# ------------------------------------------------------------------------------------------
+
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2609_09721_b200 import binding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device (the CUDA path has no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    dev = torch.device("cuda", local_rank)
+    binding.lib()
+
+    case = workload_case(args.workload)
+    qb, kb, vb = inputs.make_qkv(case)     # every rank: its own replica of the workload (weak scaling, no exchange)
+    pin = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).pin_memory()
+    hq, hk, hv = pin(qb), pin(kb), pin(vb)
+    dq, dk, dv = hq.to(dev), hk.to(dev), hv.to(dev)
+    shape = (case.B, case.Hq, case.Hkv, case.Sq, case.Sk, case.d)
+    o = torch.empty((case.B, case.Hq, case.Sq, case.d), dtype=torch.float32, device=dev)
+    ws = torch.empty(binding.efq_attention_workspace_bytes(*shape), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def step(producer=0, ev=None):
+        binding.efq_quantize_qkv(dq, dk, dv, ws)
+        if ev is not None:
+            ev[0].record(stream)
+        binding.efq_attention_fwd_quantized(o, shape, ws, case.causal, 0.0, producer)
+        if ev is not None:
+            ev[1].record(stream)
+
+    def timed(producer, steps, warmup, sampler=None):
+        for _ in range(warmup):
+            step(producer)
+        barrier()
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if sampler:
+            sampler.start()
+            time.sleep(0.25)
+        t0 = time.time()
+        e0.record(stream)
+        for i in range(steps):
+            step(producer, evs[i])
+        e1.record(stream)
+        barrier()
+        t1 = time.time()
+        clocks = sampler.stop(t0, t1) if sampler else None
+        ms = e0.elapsed_time(e1)
+        main_ms = sum(a.elapsed_time(b) for a, b in evs) / steps
+        if world > 1:
+            t = torch.tensor([ms, main_ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms, main_ms = float(t[0]), float(t[1])
+        return ms / steps, main_ms, clocks
+
+    phys_gpu = local_rank
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            phys_gpu = int(vis.split(",")[local_rank])
+        except (ValueError, IndexError):
+            phys_gpu = local_rank
+    sampler = ClockSampler(phys_gpu) if rank == 0 else None
+    ms_step, ms_main, clocks = timed(0, args.steps, args.warmup, sampler)
+    status = binding.efq_poll_status(ws)
+    if status != 0:
+        raise SystemExit(f"bench.py: device status {status} after the timed region")
+    etq_ms_step, etq_ms_main, _ = timed(1, max(3, args.steps // 2), 3)
+
+    # end to end: pinned host inputs -> device -> forward -> host output, every step
+    ho = torch.empty((case.B, case.Hq, case.Sq, case.d), dtype=torch.float32).pin_memory()
+    e2e_steps = max(3, min(args.steps, 10))
+    for _ in range(2):
+        binding.efq_attention_fwd_host(hq, hk, hv, ho, dq, dk, dv, o, case.causal, 0.0, 0, None, ws)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        binding.efq_attention_fwd_host(hq, hk, hv, ho, dq, dk, dv, o, case.causal, 0.0, 0, None, ws)
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    if world > 1:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t[0])
+    h2d = hq.numel() * 2 + hk.numel() * 2 + hv.numel() * 2
+    d2h = ho.numel() * 4
+
+    # standalone probability-generation stage (HBM-bound): EFQ vs exp-then-quantize, 4096 x 16384 fp32
+    stage = None
+    if rank == 0 and not args.skip_stage:
+        rows, cols = 4096, 16384
+        g = torch.Generator(device=dev)
+        g.manual_seed(2)
+        sc = torch.randn((rows, cols), generator=g, device=dev, dtype=torch.float32) * 3.0
+        rm = sc.max(dim=1).values.contiguous()
+        codes = torch.empty((rows, cols // 2), dtype=torch.uint8, device=dev)
+        scl = torch.empty((rows, cols // 32), dtype=torch.uint8, device=dev)
+        nbytes = rows * cols * (4 + 0.5 + 1 / 32)
+
+        def stage_time(fn):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(20):
+                fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / 20
+
+        t_efq = stage_time(lambda: binding.efq_probgen(sc, rm, 1.0, None, codes, scl))
+        t_etq = stage_time(lambda: binding.exp_then_quantize_probgen(sc, rm, 1.0, 0, codes, scl))
+        stage = {"workload": "probgen 4096x16384 fp32 (device-generated N(0,9), timing only)", "bytes_per_launch": nbytes,
+                 "efq_ms": t_efq, "efq_gbs": nbytes / t_efq / 1e6, "etq_ms": t_etq, "etq_gbs": nbytes / t_etq / 1e6}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    flops = case.flops
+    value = world * flops / (ms_step * 1e-3) / 1e12
+    main_tflops = flops / (ms_main * 1e-3) / 1e12
+    fp4_peak = peaks["bf16_sustained"] * NOMINAL_FP4_OVER_BF16
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "attention_fwd_traffic.json")
+    if os.path.exists(tpath):
+        with open(tpath) as f:
+            traffic = json.load(f).get(args.workload)
+
+    cpu_baseline = None
+    if world == 1 and not args.skip_cpu_baseline:
+        q32, k32, v32 = (inputs.bf16_bits_to_f32(t) for t in (qb, kb, vb))
+        n_rows = args.oracle_rows
+        cv, csec, cores = time_oracle(case, q32, k32, v32, n_rows, 3, 1)
+        cpu_baseline = {"value": cv, "unit": UNIT, "cores": cores, "kind": "oracle",
+                        "sample": f"3 steps of {n_rows} seeded query rows (all heads), EFQ path, {csec:.2f} s per step"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp4_e2m1",
+        "data": "synthetic",
+        "config": {"workload": case.name, "B": case.B, "Hq": case.Hq, "Hkv": case.Hkv, "S": case.Sq, "d": case.d,
+                   "causal": case.causal, "kv_tile": 128, "params": "EFQ-Mean tau=-3.06 h=2.30",
+                   "l2": "inputs larger than L2 (Q+K+V bf16 and fp32 O exceed 126 MB)", "parallelism": f"replicas x{world}"},
+        "clocks": clocks,
+        "e2e": {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+        "gpu_launches": 4 * args.steps,
+        "roofline": {"kernel": "attention_fwd_kernel<EFQ>", "bound": "tensor", "achieved": main_tflops, "peak": fp4_peak,
+                     "unit": "TFLOP/s", "frac": main_tflops / fp4_peak, "traffic": traffic,
+                     "peak_source": f"{peaks['source']} bf16 sustained {peaks['bf16_sustained']} TFLOP/s x {NOMINAL_FP4_OVER_BF16} "
+                                    "(nominal FP4:bf16 ratio)", "ms_per_launch": ms_main,
+                     "frac_of_nominal_9pflops": main_tflops / 9000.0},
+        "cpu_baseline": cpu_baseline,
+        "exp_then_quantize": {"value": flops / (etq_ms_step * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": etq_ms_step,
+                              "main_kernel_ms": etq_ms_main, "efq_speedup": etq_ms_step / ms_step},
+        "stage": stage,
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="qwen3_8b_16k")
+    ap.add_argument("--oracle-rows", type=int, default=512)
+    ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--skip-stage", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()
