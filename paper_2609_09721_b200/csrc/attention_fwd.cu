@@ -8,7 +8,7 @@
 //               S_j = Q^ K^_j^T  and  [dA | dl] = P~_j [V^_j | 1]  as kind::mxf4 block-scaled MMAs,
 //               FP32 accumulators in TMEM.  The 16 "ones" rows appended to V^T give the denominator
 //               P~1 from the very operand that feeds the numerator.
-//   warps 2-9   probability generation: thread = (query row, half of the 128 keys).  Scores come
+//   warps 4-11  probability generation: thread = (query row, half of the 128 keys).  Scores come
 //               from TMEM straight into registers; block maxima and the running row maximum are
 //               thread-local plus one shared-memory exchange between the two halves; codes go as
 //               16-byte packed stores into the swizzled shared-memory A operand, scale bytes into
@@ -36,7 +36,7 @@ namespace {
 
 constexpr int kTile = 128;            // query rows per CTA and keys per KV tile (Bc)
 constexpr int kStages = 3;            // K and V ring depth
-constexpr int kThreads = 320;         // 10 warps
+constexpr int kThreads = 384;         // 12 warps = 3 warpgroups: {TMA, MMA, 2 idle}, 2 x probability generation
 constexpr int kSoftmaxWarps = 8;
 constexpr int kTileBytes = kTile * 64;          // 128 rows x 64 B of packed E2M1
 constexpr int kSfBytes = 512;
@@ -116,8 +116,47 @@ __device__ __forceinline__ uint32_t p_swizzled_offset(uint32_t row, uint32_t chu
     return (row >> 3) * 512u + (row & 7u) * 64u + ((chunk ^ ((row >> 1) & 3u)) << 4);
 }
 
-// 32 scores of one microscaling block -> 16 bytes of codes + scale byte (EFQ: Algorithm 1).
-template <int PRODUCER>
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float fma_sat(float a, float b, float c)
+{
+    float d;
+    asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t pack2(float lo, float hi)
+{
+    uint64_t d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+    return d;
+}
+
+// Largest of 32 scores with 3-input maxima.
+__device__ __forceinline__ float block_max32(const float* r)
+{
+    float m[11];
+#pragma unroll
+    for (int i = 0; i < 10; ++i) m[i] = max3(r[3 * i], r[3 * i + 1], r[3 * i + 2]);
+    m[10] = fmaxf(r[30], r[31]);
+    const float a = max3(m[0], m[1], m[2]), b = max3(m[3], m[4], m[5]), c = max3(m[6], m[7], m[8]);
+    return max3(max3(a, b, c), m[9], m[10]);
+}
+
+// 32 scores of one microscaling block -> 16 bytes of codes + scale byte.
+//
+// EFQ (Algorithm 1), three FMA-pipe instructions per element, bit-identical to
+// c = floor(min(max(fma(r, A, Bb), 0), 7)):
+//   w  = fma.rn.sat(r, A/8, Bb/8)      = clamp(fma(r, A, Bb), 0, 8) / 8   (scaling by 2^-3 commutes with rounding)
+//   a' = fma.rm(w, 8, u)               = u + floor(8 w)                   (u an integer in [2^23, 2^24): ulp 1, round down)
+//   u' = fma.rn(a', 16, -15 * 2^23)    = 2^23 + 16 X                      (a' = 2^23 + X, exact)
+// so four elements accumulate Horner-style into X = c3 c2 c1 c0 (one nibble each) in the mantissa; the two
+// chain steps run as packed f32x2 FMAs on the low and high half of a 32-bit word at once.  floor(8 w) = 8 happens
+// only when fma(r, A, Bb) >= 8; FIX8 turns that nibble into 7 (needed when (ln 1.5 - tau) h + 1 can reach 8).
+template <int PRODUCER, bool FIX8>
 __device__ __forceinline__ void produce32(const float* r, float rmax, float m_s, const ProducerConsts& K, uint4& codes,
                                           uint32_t& byte)
 {
@@ -125,11 +164,23 @@ __device__ __forceinline__ void produce32(const float* r, float rmax, float m_s,
     if (PRODUCER == 0) {
         BlockScale s = efq_block_scale(rmax, m_s, K);
         byte = s.byte;
+        const float A8 = K.A * 0.125f, B8 = s.Bb * 0.125f;
+        const uint64_t eight2 = pack2(8.0f, 8.0f), sixteen2 = pack2(16.0f, 16.0f);
+        const uint64_t magic2 = pack2(8388608.0f, 8388608.0f), back2 = pack2(-125829120.0f, -125829120.0f);
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-            uint32_t word = 0;
+            uint64_t a2 = magic2;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) word |= efq_code(r[q * 8 + i], K.A, s.Bb) << (4 * i);
+            for (int i = 3; i >= 0; --i) {
+                const uint64_t w2 = pack2(fma_sat(r[q * 8 + i], A8, B8), fma_sat(r[q * 8 + 4 + i], A8, B8));
+                uint64_t u2 = magic2;
+                if (i != 3) asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(u2) : "l"(a2), "l"(sixteen2), "l"(back2));
+                asm("fma.rm.f32x2 %0, %1, %2, %3;" : "=l"(a2) : "l"(w2), "l"(eight2), "l"(u2));
+            }
+            uint32_t lo, hi;
+            asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(a2));
+            uint32_t word = __byte_perm(lo, hi, 0x5410);
+            if (FIX8) word -= (word >> 3) & 0x11111111u;
             w[q] = s.live ? word : 0u;
         }
     } else {
@@ -164,7 +215,7 @@ __device__ __forceinline__ void produce32(const float* r, float rmax, float m_s,
     codes = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-template <int PRODUCER, bool DEBUG>
+template <int PRODUCER, bool DEBUG, bool FIX8>
 __global__ void __launch_bounds__(kThreads, 1)
 attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                      const __grid_constant__ CUtensorMap map_v, const FwdParams P)
@@ -225,6 +276,9 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     const uint32_t tmem = sm->tmem_base;
     const bool run = sm->abort_flag == 0 && n_tiles > 0;
 
+    // register budget: the probability warpgroups take what the producer/issuer warpgroup gives up
+    if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
     if (run && warp == 0) {
         // =============================== TMA producer ===============================
         if (lane == 0) {
@@ -286,10 +340,13 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             __syncwarp();
             return true;
         };
+        // S runs two tiles ahead of P~V so that the next tile's scores are in TMEM before the
+        // probability warps finish the current one.
         if (ok) ok = issue_qk(0);
+        if (ok && n_tiles > 1) ok = issue_qk(1);
         for (int64_t j = 0; ok && j < n_tiles; ++j) {
-            if (j + 1 < n_tiles) {
-                ok = issue_qk(j + 1);
+            if (j + 2 < n_tiles) {
+                ok = issue_qk(j + 2);
                 if (!ok) break;
             }
             const int s = static_cast<int>(j % kStages);
@@ -317,10 +374,13 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             }
             __syncwarp();
         }
-    } else if (run && warp >= 2) {
+    }
+    } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+    if (run) {
         // =============================== probability generation ===============================
         const int quarter = warp & 3;                       // TMEM lane quarter this warp may touch
-        const int half = (warp - 2) >> 2;                   // which 64 keys of the tile
+        const int half = (warp - 4) >> 2;                   // which 64 keys of the tile
         const uint32_t row = quarter * 32 + lane;           // row inside the query tile
         const int64_t grow = q0 + row;                      // global query row
         const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
@@ -336,10 +396,13 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         float m_raw = -INFINITY;
         float m_s = -INFINITY;
         bool ok = true;
-        for (int64_t j = 0; j < n_tiles; ++j) {
-            const int sb = static_cast<int>(j & 1);
-            const uint32_t ph2 = static_cast<uint32_t>((j >> 1) & 1);
-            if (!wait_barrier(&sm->s_full[sb], ph2, sm, P.status)) { ok = false; break; }
+
+        // Scores of tile t: TMEM -> registers (this thread's 64 keys), masked, with the two block maxima;
+        // the half-row maximum is published for the partner thread that owns the other 64 keys of the row.
+        auto fetch = [&](int64_t t, float (&r)[64], float (&bmax)[2]) -> bool {
+            const int sb = static_cast<int>(t & 1);
+            const uint32_t ph2 = static_cast<uint32_t>((t >> 1) & 1);
+            if (!wait_barrier(&sm->s_full[sb], ph2, sm, P.status)) return false;
             ptx::tc_fence_after_sync();
             uint32_t sr[64];
             const uint32_t s_addr = tmem + lane_base + kColS + 128 * sb + 64 * half;
@@ -349,31 +412,33 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&sm->s_empty[sb]);
-
-            float r[64];
-            const int64_t key0 = j * kTile + 64 * half;
-            const bool need_mask = key0 + 63 > limit;
+            const int64_t key0 = t * kTile + 64 * half;
+            if (key0 + 63 > limit) {
 #pragma unroll
-            for (int i = 0; i < 64; ++i) {
-                r[i] = __uint_as_float(sr[i]);
-                if (need_mask && key0 + i > limit) r[i] = -INFINITY;
+                for (int i = 0; i < 64; ++i) r[i] = key0 + i > limit ? -INFINITY : __uint_as_float(sr[i]);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 64; ++i) r[i] = __uint_as_float(sr[i]);
             }
-            float bmax[2];
-#pragma unroll
-            for (int g = 0; g < 2; ++g) {
-                float m = r[g * 32];
-#pragma unroll
-                for (int i = 1; i < 32; ++i) m = fmaxf(m, r[g * 32 + i]);
-                bmax[g] = m;
-            }
-            // running row maximum (Eq. rowmax-update): exchange the two halves' maxima
-            const float mine = fmaxf(bmax[0], bmax[1]);
-            sm->xchg[sb][half][row] = mine;
+            bmax[0] = block_max32(&r[0]);
+            bmax[1] = block_max32(&r[32]);
+            sm->xchg[sb][half][row] = fmaxf(bmax[0], bmax[1]);
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&sm->x_bar[sb][quarter]);
-            if (!wait_barrier(&sm->x_bar[sb][quarter], ph2, sm, P.status)) { ok = false; break; }
+            return true;
+        };
+
+        // One KV tile (Algorithm 2, steps 2-13 for this thread's half row); `nxt` is filled for tile j+1 first so
+        // that its maximum exchange overlaps this tile's code generation.
+        auto body = [&](int64_t j, float (&cur)[64], float (&cmax)[2], float (&nxt)[64], float (&nmax)[2]) -> bool {
+            const int sb = static_cast<int>(j & 1);
+            const uint32_t ph2 = static_cast<uint32_t>((j >> 1) & 1);
+            if (j + 1 < n_tiles && !fetch(j + 1, nxt, nmax)) return false;
+
+            // running row maximum (Eq. rowmax-update) with the partner's half
+            if (!wait_barrier(&sm->x_bar[sb][quarter], ph2, sm, P.status)) return false;
             const float other = sm->xchg[sb][half ^ 1][row];
-            const float m_new = fmaxf(m_raw, fmaxf(mine, other));
+            const float m_new = fmaxf(m_raw, max3(cmax[0], cmax[1], other));
             const float m_s_new = __fmul_rn(K.sigma, m_new);
             const bool grew = m_new > m_raw && m_raw != -INFINITY;   // history exists and must be rescaled
             const float alpha = grew ? ex2_approx(__fmul_rn(__fsub_rn(m_s, m_s_new), K.LOG2E)) : 1.0f;
@@ -381,12 +446,13 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             m_s = m_s_new;
 
             // P buffer sb free?  (P~V of tile j-2 finished)
-            if (!wait_barrier(&sm->p_empty[sb], ph2 ^ 1u, sm, P.status)) { ok = false; break; }
+            if (!wait_barrier(&sm->p_empty[sb], ph2 ^ 1u, sm, P.status)) return false;
+            const int64_t key0 = j * kTile + 64 * half;
             uint32_t bytes[2];
 #pragma unroll
             for (int g = 0; g < 2; ++g) {
                 uint4 codes;
-                produce32<PRODUCER>(&r[g * 32], bmax[g], m_s, K, codes, bytes[g]);
+                produce32<PRODUCER, FIX8>(&cur[g * 32], cmax[g], m_s, K, codes, bytes[g]);
                 if (m_new == -INFINITY) { codes = make_uint4(0, 0, 0, 0); bytes[g] = 0; }
                 *reinterpret_cast<uint4*>(sm->p[sb] + p_swizzled_offset(row, 2 * half + g)) = codes;
                 if (DEBUG && dbg_row) {
@@ -402,7 +468,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             if (DEBUG && dbg_row) {
                 if (P.dbg.raw_scores) {
                     for (int i = 0; i < 64; ++i)
-                        if (key0 + i < P.Sk) P.dbg.raw_scores[drow * P.Sk + key0 + i] = r[i];
+                        if (key0 + i < P.Sk) P.dbg.raw_scores[drow * P.Sk + key0 + i] = cur[i];
                 }
                 if (P.dbg.row_max && half == 0) P.dbg.row_max[drow * ntile_all + j] = m_s;
             }
@@ -410,7 +476,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             // historical rescaling (Eq. alpha): O rows and the denominator column in TMEM
             if (j > 0 && __any_sync(0xffffffffu, grew)) {
                 const int pv = static_cast<int>((j - 1) & 1);
-                if (!wait_barrier(&sm->p_empty[pv], static_cast<uint32_t>(((j - 1) >> 1) & 1), sm, P.status)) { ok = false; break; }
+                if (!wait_barrier(&sm->p_empty[pv], static_cast<uint32_t>(((j - 1) >> 1) & 1), sm, P.status)) return false;
                 ptx::tc_fence_after_sync();
                 uint32_t o[64];
                 const uint32_t o_addr = tmem + lane_base + kColO + 64 * half;
@@ -430,6 +496,16 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&sm->p_full[sb]);
+            return true;
+        };
+
+        {
+            float ra[64], rb[64], ma[2], mb[2];
+            ok = fetch(0, ra, ma);
+            for (int64_t j = 0; ok && j < n_tiles; j += 2) {
+                ok = body(j, ra, ma, rb, mb);
+                if (ok && j + 1 < n_tiles) ok = body(j + 1, rb, mb, ra, ma);
+            }
         }
         // ---- final normalisation O = A / l
         if (ok) {
@@ -459,14 +535,15 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 }
             }
         }
-    } else if (!run && warp >= 2 && sm->abort_flag == 0) {
+    } else if (sm->abort_flag == 0) {
         // no visible key for the whole tile: rows are zero
-        const int quarter = warp & 3, half = (warp - 2) >> 2;
+        const int quarter = warp & 3, half = (warp - 4) >> 2;
         const int64_t grow = q0 + quarter * 32 + lane;
         if (grow < P.Sq) {
             float4* dst = reinterpret_cast<float4*>(P.o + ((bh * P.Sq + grow) * 128 + 64 * half));
             for (int i = 0; i < 16; ++i) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
+    }
     }
 
     ptx::tc_fence_before_sync();
@@ -540,21 +617,26 @@ bool shape_ok(int B, int Hq, int Hkv, int64_t Sq, int64_t Sk, int d)
            static_cast<int64_t>(B) * Hkv * ((Sk + kTile - 1) / kTile * kTile) < (1ll << 31);
 }
 
-template <int PRODUCER>
-cudaError_t launch_main(bool debug, dim3 grid, size_t smem, cudaStream_t stream, const CUtensorMap& mq, const CUtensorMap& mk,
-                        const CUtensorMap& mv, const FwdParams& P)
+template <int PRODUCER, bool DEBUG, bool FIX8>
+cudaError_t launch_one(dim3 grid, size_t smem, cudaStream_t stream, const CUtensorMap& mq, const CUtensorMap& mk,
+                       const CUtensorMap& mv, const FwdParams& P)
 {
-    cudaError_t e;
-    if (debug) {
-        e = cudaFuncSetAttribute(attention_fwd_kernel<PRODUCER, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-        if (e != cudaSuccess) return e;
-        attention_fwd_kernel<PRODUCER, true><<<grid, kThreads, smem, stream>>>(mq, mk, mv, P);
-    } else {
-        e = cudaFuncSetAttribute(attention_fwd_kernel<PRODUCER, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-        if (e != cudaSuccess) return e;
-        attention_fwd_kernel<PRODUCER, false><<<grid, kThreads, smem, stream>>>(mq, mk, mv, P);
-    }
+    cudaError_t e = cudaFuncSetAttribute(attention_fwd_kernel<PRODUCER, DEBUG, FIX8>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    attention_fwd_kernel<PRODUCER, DEBUG, FIX8><<<grid, kThreads, smem, stream>>>(mq, mk, mv, P);
     return cudaGetLastError();
+}
+
+template <int PRODUCER>
+cudaError_t launch_main(bool debug, bool fix8, dim3 grid, size_t smem, cudaStream_t stream, const CUtensorMap& mq,
+                        const CUtensorMap& mk, const CUtensorMap& mv, const FwdParams& P)
+{
+    if (PRODUCER != 0) fix8 = false;
+    if (debug) return fix8 ? launch_one<PRODUCER, true, true>(grid, smem, stream, mq, mk, mv, P)
+                           : launch_one<PRODUCER, true, false>(grid, smem, stream, mq, mk, mv, P);
+    return fix8 ? launch_one<PRODUCER, false, true>(grid, smem, stream, mq, mk, mv, P)
+                : launch_one<PRODUCER, false, false>(grid, smem, stream, mq, mk, mv, P);
 }
 
 efq_status_t attention_impl(const void* q, const void* k, const void* v, float* o, int B, int Hq, int Hkv, int64_t Sq,
@@ -608,11 +690,13 @@ efq_status_t attention_impl(const void* q, const void* k, const void* v, float* 
     dim3 grid(static_cast<unsigned>(items));
     // more than half of the SM's shared memory: one CTA per SM, since each CTA takes all 512 TMEM columns
     const size_t smem = sizeof(Smem) + 1024 > 120 * 1024 ? sizeof(Smem) + 1024 : 120 * 1024;
+    // fma(r, A, Bb) can reach 8 only if the residual of a block maximum, below ln 1.5, maps that high
+    const bool fix8 = (log(1.5) - static_cast<double>(tau)) * static_cast<double>(h) + 1.0 > 7.999;
     cudaError_t e;
     switch (producer) {
-        case 0: e = launch_main<0>(debug != nullptr, grid, smem, stream, mq, mk, mv, P); break;
-        case 1: e = launch_main<1>(debug != nullptr, grid, smem, stream, mq, mk, mv, P); break;
-        case 2: e = launch_main<2>(debug != nullptr, grid, smem, stream, mq, mk, mv, P); break;
+        case 0: e = launch_main<0>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
+        case 1: e = launch_main<1>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
+        case 2: e = launch_main<2>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
         default: return EFQ_ERR_INVALID_ARG;
     }
     return e == cudaSuccess ? EFQ_OK : EFQ_ERR_CUDA;
