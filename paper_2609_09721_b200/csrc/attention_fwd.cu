@@ -3,16 +3,18 @@
 //
 // One CTA owns one 128-row query tile of one (batch, head) and walks the KV tiles of width 128:
 //   warp 0      TMA producer: Q tile once, then K_j / V^T_j code tiles (SW64 layout) and their
-//               512-byte scale tiles through 3-stage mbarrier rings
+//               512-byte scale tiles through 4-stage mbarrier rings
 //   warp 1      MMA issuer (one elected thread): scale tiles smem -> TMEM (tcgen05.cp), then
 //               S_j = Q^ K^_j^T  and  [dA | dl] = P~_j [V^_j | 1]  as kind::mxf4 block-scaled MMAs,
 //               FP32 accumulators in TMEM.  The 16 "ones" rows appended to V^T give the denominator
 //               P~1 from the very operand that feeds the numerator.
-//   warps 4-11  probability generation: thread = (query row, half of the 128 keys).  Scores come
-//               from TMEM straight into registers; block maxima and the running row maximum are
-//               thread-local plus one shared-memory exchange between the two halves; codes go as
-//               16-byte packed stores into the swizzled shared-memory A operand, scale bytes into
-//               the scale tile.  No FP16/FP32 probability tile exists anywhere.
+//   warps 4-11  probability generation, two groups of four warps: group 0 takes the even KV tiles,
+//               group 1 the odd ones, so one group's latency-bound steps (TMEM load, hand-over of the
+//               running maximum, accumulator rescaling) overlap the other group's code generation.
+//               Thread = query row: the 128 scores of the row come from TMEM straight into registers;
+//               block maxima, scale and codes are thread-local; codes go as 16-byte packed stores into
+//               the swizzled shared-memory A operand, the four scale bytes as one word into the scale
+//               tile.  No FP16/FP32 probability tile exists anywhere.
 // The online recurrence is unchanged: when a row's maximum grows, the accumulator rows in TMEM
 // are rescaled by alpha = exp(m_old - m_new) before the next P~V MMA is released.
 //
@@ -32,12 +34,20 @@ cudaError_t launch_quantize_rows(const void* x, int64_t n_heads, int64_t S, int6
 cudaError_t launch_quantize_v(const void* v, int64_t n_heads, int64_t S, int64_t S_pad, uint8_t* vt_codes, uint8_t* sf,
                               cudaStream_t stream);
 
+#ifdef EFQ_TIMELINE
+__device__ long long* g_timeline = nullptr;   // [role 0..2][tile][8] clock stamps of CTA 0 (working instrumentation)
+#define TL(role, tile, slot) do { if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && g_timeline && (tile) < 256) \
+    g_timeline[((role) * 256 + (tile)) * 8 + (slot)] = clock64(); } while (0)
+#else
+#define TL(role, tile, slot) do { } while (0)
+#endif
+
 namespace {
 
 constexpr int kTile = 128;            // query rows per CTA and keys per KV tile (Bc)
-constexpr int kStages = 3;            // K and V ring depth
+constexpr int kStages = 4;            // K and V ring depth
 constexpr int kThreads = 384;         // 12 warps = 3 warpgroups: {TMA, MMA, 2 idle}, 2 x probability generation
-constexpr int kSoftmaxWarps = 8;
+constexpr int kGroupWarps = 4;        // warps per probability group (one thread per query row)
 constexpr int kTileBytes = kTile * 64;          // 128 rows x 64 B of packed E2M1
 constexpr int kSfBytes = 512;
 constexpr int kVStageBytes = kTileBytes + 1024; // + 16 ones rows
@@ -62,13 +72,14 @@ struct __align__(1024) Smem {
     uint8_t sf_v[kStages][kSfBytes];
     uint8_t sf_p[2][kSfBytes];
     uint8_t sf_ones[kSfBytes];
-    float xchg[2][2][kTile];
+    float runmax[2][kTile];   // running row maximum after the group's latest tile, raw score units
     uint64_t q_full;
     uint64_t k_full[kStages], k_empty[kStages];
     uint64_t v_full[kStages], v_empty[kStages];
     uint64_t s_full[2], s_empty[2];
     uint64_t p_full[2], p_empty[2];
-    uint64_t x_bar[2][4];   // row-maximum exchange between the two halves of a lane quarter
+    uint64_t x_bar[2][4];     // [group][lane quarter]: runmax of the group's latest tile is published
+    uint64_t o_done;          // the last P~V of the work item has completed
     uint32_t tmem_base;
     volatile uint32_t abort_flag;
 };
@@ -88,27 +99,26 @@ struct FwdParams {
     int has_dbg;
 };
 
-// Warp-collective bounded wait: lane 0 polls, the verdict is broadcast.  Returns false on timeout/abort.
-__device__ __forceinline__ bool wait_barrier(uint64_t* bar, uint32_t parity, Smem* sm, uint32_t* status)
+// Bounded wait of one thread.  Returns false on timeout (recorded in the status word) or CTA-wide abort.
+__device__ __forceinline__ bool wait1(uint64_t* bar, uint32_t parity, Smem* sm, uint32_t* status)
 {
-    uint32_t ok = 1;
-    if ((threadIdx.x & 31) == 0) {
-        if (!ptx::mbar_try_wait(bar, parity)) {
-            const long long t0 = clock64();
-            while (true) {
-                if (ptx::mbar_try_wait(bar, parity)) break;
-                if (sm->abort_flag) { ok = 0; break; }
-                if (static_cast<uint64_t>(clock64() - t0) > kTimeoutCycles) {
-                    ok = 0;
-                    sm->abort_flag = 1;
-                    atomicExch(status, static_cast<uint32_t>(EFQ_ERR_DEVICE_TIMEOUT));
-                    break;
-                }
-            }
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (true) {
+        if (ptx::mbar_try_wait_suspend(bar, parity, 20000u)) return true;
+        if (sm->abort_flag) return false;
+        if (static_cast<uint64_t>(clock64() - t0) > kTimeoutCycles) {
+            sm->abort_flag = 1;
+            atomicExch(status, static_cast<uint32_t>(EFQ_ERR_DEVICE_TIMEOUT));
+            return false;
         }
     }
-    ok = __shfl_sync(0xffffffffu, ok, 0);
-    return ok != 0;
+}
+// The same wait executed by all lanes of a warp; the verdict is made warp-uniform.
+__device__ __forceinline__ bool wait_all(uint64_t* bar, uint32_t parity, Smem* sm, uint32_t* status)
+{
+    const bool ok = wait1(bar, parity, sm, status);
+    return __all_sync(0xffffffffu, ok);
 }
 
 __device__ __forceinline__ uint32_t p_swizzled_offset(uint32_t row, uint32_t chunk)
@@ -247,6 +257,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     // ---- setup
     if (threadIdx.x == 0) {
         ptx::mbar_init(&sm->q_full, 1);
+        ptx::mbar_init(&sm->o_done, 1);
         for (int s = 0; s < kStages; ++s) {
             ptx::mbar_init(&sm->k_full[s], 1);
             ptx::mbar_init(&sm->k_empty[s], 1);
@@ -255,10 +266,10 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         }
         for (int i = 0; i < 2; ++i) {
             ptx::mbar_init(&sm->s_full[i], 1);
-            ptx::mbar_init(&sm->s_empty[i], kSoftmaxWarps);
-            ptx::mbar_init(&sm->p_full[i], kSoftmaxWarps);
+            ptx::mbar_init(&sm->s_empty[i], kGroupWarps);
+            ptx::mbar_init(&sm->p_full[i], kGroupWarps);
             ptx::mbar_init(&sm->p_empty[i], 1);
-            for (int qd = 0; qd < 4; ++qd) ptx::mbar_init(&sm->x_bar[i][qd], 2);
+            for (int qd = 0; qd < 4; ++qd) ptx::mbar_init(&sm->x_bar[i][qd], 1);
         }
         sm->abort_flag = (*reinterpret_cast<volatile uint32_t*>(P.status) != 0u) ? 1u : 0u;
         ptx::mbar_init_fence();
@@ -279,111 +290,99 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     // register budget: the probability warpgroups take what the producer/issuer warpgroup gives up
     if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
-    if (run && warp == 0) {
-        // =============================== TMA producer ===============================
-        if (lane == 0) {
-            ptx::mbar_arrive_expect_tx(&sm->q_full, kTileBytes + kSfBytes);
-            ptx::tma_load_2d(sm->q, &map_q, 0, static_cast<int>(bh * P.Sq_pad + q0), &sm->q_full);
-            ptx::bulk_load_1d(sm->sf_q, P.sf_q + (bh * n_qtiles + qt) * kSfBytes, kSfBytes, &sm->q_full);
-        }
+    if (run && warp == 0 && lane == 0) {
+        // =============================== TMA producer (one thread) ===============================
+        ptx::mbar_arrive_expect_tx(&sm->q_full, kTileBytes + kSfBytes);
+        ptx::tma_load_2d(sm->q, &map_q, 0, static_cast<int>(bh * P.Sq_pad + q0), &sm->q_full);
+        ptx::bulk_load_1d(sm->sf_q, P.sf_q + (bh * n_qtiles + qt) * kSfBytes, kSfBytes, &sm->q_full);
         const int64_t kvh = static_cast<int64_t>(b) * P.Hkv + hkv;
         const int64_t kv_tiles = P.Sk_pad / kTile;
+        int s = 0;
+        uint32_t ph = 0;
         for (int64_t j = 0; j < n_tiles; ++j) {
-            const int s = static_cast<int>(j % kStages);
-            const uint32_t ph = static_cast<uint32_t>((j / kStages) & 1);
-            if (!wait_barrier(&sm->k_empty[s], ph ^ 1u, sm, P.status)) break;
-            if (lane == 0) {
-                ptx::mbar_arrive_expect_tx(&sm->k_full[s], kTileBytes + kSfBytes);
-                ptx::tma_load_2d(sm->k[s], &map_k, 0, static_cast<int>(kvh * P.Sk_pad + j * kTile), &sm->k_full[s]);
-                ptx::bulk_load_1d(sm->sf_k[s], P.sf_k + (kvh * kv_tiles + j) * kSfBytes, kSfBytes, &sm->k_full[s]);
-            }
-            if (!wait_barrier(&sm->v_empty[s], ph ^ 1u, sm, P.status)) break;
-            if (lane == 0) {
-                ptx::mbar_arrive_expect_tx(&sm->v_full[s], kTileBytes + kSfBytes);
-                ptx::tma_load_2d(sm->v[s], &map_v, static_cast<int>(j * 64), static_cast<int>(kvh * 128), &sm->v_full[s]);
-                ptx::bulk_load_1d(sm->sf_v[s], P.sf_v + (kvh * kv_tiles + j) * kSfBytes, kSfBytes, &sm->v_full[s]);
-            }
+            if (!wait1(&sm->k_empty[s], ph ^ 1u, sm, P.status)) break;
+            ptx::mbar_arrive_expect_tx(&sm->k_full[s], kTileBytes + kSfBytes);
+            ptx::tma_load_2d(sm->k[s], &map_k, 0, static_cast<int>(kvh * P.Sk_pad + j * kTile), &sm->k_full[s]);
+            ptx::bulk_load_1d(sm->sf_k[s], P.sf_k + (kvh * kv_tiles + j) * kSfBytes, kSfBytes, &sm->k_full[s]);
+            if (!wait1(&sm->v_empty[s], ph ^ 1u, sm, P.status)) break;
+            ptx::mbar_arrive_expect_tx(&sm->v_full[s], kTileBytes + kSfBytes);
+            ptx::tma_load_2d(sm->v[s], &map_v, static_cast<int>(j * 64), static_cast<int>(kvh * 128), &sm->v_full[s]);
+            ptx::bulk_load_1d(sm->sf_v[s], P.sf_v + (kvh * kv_tiles + j) * kSfBytes, kSfBytes, &sm->v_full[s]);
+            if (++s == kStages) { s = 0; ph ^= 1u; }
         }
-    } else if (run && warp == 1) {
-        // =============================== MMA issuer ===============================
-        const uint32_t q_addr = ptx::smem_u32(sm->q);
-        bool ok = wait_barrier(&sm->q_full, 0, sm, P.status);
+    } else if (run && warp == 1 && lane == 0) {
+        // =============================== MMA issuer (one thread) ===============================
+        // Descriptors differ from tile to tile only in the start-address field (address >> 4).
+        const uint64_t d_sw64 = ptx::smem_desc(0, 16, 512, ptx::kLayoutSw64);
+        const uint64_t d_sf = ptx::smem_desc(0, 16, 128, ptx::kLayoutNone);
+        const uint64_t dq0 = d_sw64 + (ptx::smem_u32(sm->q) >> 4);
+        const uint32_t idesc_qk0 = ptx::mxf4_idesc(128, 0), idesc_qk1 = ptx::mxf4_idesc(128, 2);
+        const uint32_t idesc_pv0 = ptx::mxf4_idesc(144, 0), idesc_pv1 = ptx::mxf4_idesc(144, 2);
+        const uint32_t sfq = tmem + kColSfQ;
+        bool ok = wait1(&sm->q_full, 0, sm, P.status);
         ptx::tc_fence_after_sync();
-        if (ok && lane == 0) {
-            ptx::tmem_cp_sf(tmem + kColSfQ, ptx::smem_desc(ptx::smem_u32(sm->sf_q), 16, 128, ptx::kLayoutNone));
-            const uint64_t d1 = ptx::smem_desc(ptx::smem_u32(sm->sf_ones), 16, 128, ptx::kLayoutNone);
+        if (ok) {
+            ptx::tmem_cp_sf(sfq, d_sf + (ptx::smem_u32(sm->sf_q) >> 4));
+            const uint64_t d1 = d_sf + (ptx::smem_u32(sm->sf_ones) >> 4);
             ptx::tmem_cp_sf(tmem + kColSfV + 4, d1);
             ptx::tmem_cp_sf(tmem + kColSfV + 12, d1);
         }
-        // QK_j: S[j&1] = Q K_j^T
-        auto issue_qk = [&](int64_t j) -> bool {
-            const int s = static_cast<int>(j % kStages);
-            const uint32_t ph = static_cast<uint32_t>((j / kStages) & 1);
-            const int sb = static_cast<int>(j & 1);
-            if (!wait_barrier(&sm->k_full[s], ph, sm, P.status)) return false;
-            if (!wait_barrier(&sm->s_empty[sb], static_cast<uint32_t>((j >> 1) & 1) ^ 1u, sm, P.status)) return false;
+        int ks = 0;                 // K ring position of the next QK to issue
+        uint32_t kph = 0;
+        int64_t next_qk = 0;
+        // QK_t: S[t&1] = Q K_t^T
+        auto issue_qk = [&]() -> bool {
+            const int64_t t = next_qk;
+            const int sb = static_cast<int>(t & 1);
+            if (!wait1(&sm->k_full[ks], kph, sm, P.status)) return false;
+            if (!wait1(&sm->s_empty[sb], static_cast<uint32_t>((t >> 1) & 1) ^ 1u, sm, P.status)) return false;
             ptx::tc_fence_after_sync();
-            if (lane == 0) {
-                const uint32_t sfk = tmem + kColSfK + 4 * sb;
-                ptx::tmem_cp_sf(sfk, ptx::smem_desc(ptx::smem_u32(sm->sf_k[s]), 16, 128, ptx::kLayoutNone));
-                const uint32_t k_addr = ptx::smem_u32(sm->k[s]);
-#pragma unroll
-                for (uint32_t kk = 0; kk < 2; ++kk) {
-                    const uint32_t id = kk * 2;
-                    ptx::mma_mxf4(tmem + kColS + 128 * sb, ptx::smem_desc(q_addr + 32 * kk, 16, 512, ptx::kLayoutSw64),
-                                  ptx::smem_desc(k_addr + 32 * kk, 16, 512, ptx::kLayoutSw64), ptx::mxf4_idesc(128, id),
-                                  (tmem + kColSfQ) | (id << 30), sfk | (id << 30), kk);
-                }
-                ptx::mma_commit(&sm->k_empty[s]);
-                ptx::mma_commit(&sm->s_full[sb]);
-            }
-            __syncwarp();
+            const uint32_t sfk = tmem + kColSfK + 4 * sb;
+            ptx::tmem_cp_sf(sfk, d_sf + (ptx::smem_u32(sm->sf_k[ks]) >> 4));
+            const uint64_t dk0 = d_sw64 + (ptx::smem_u32(sm->k[ks]) >> 4);
+            const uint32_t d_s = tmem + kColS + 128 * sb;
+            ptx::mma_mxf4(d_s, dq0, dk0, idesc_qk0, sfq, sfk, 0u);
+            ptx::mma_mxf4(d_s, dq0 + 2, dk0 + 2, idesc_qk1, sfq | (2u << 30), sfk | (2u << 30), 1u);
+            ptx::mma_commit(&sm->k_empty[ks]);
+            ptx::mma_commit(&sm->s_full[sb]);
+            if (++ks == kStages) { ks = 0; kph ^= 1u; }
+            ++next_qk;
             return true;
         };
-        // S runs two tiles ahead of P~V so that the next tile's scores are in TMEM before the
-        // probability warps finish the current one.
-        if (ok) ok = issue_qk(0);
-        if (ok && n_tiles > 1) ok = issue_qk(1);
+        // S runs two tiles ahead of P~V so that a tile's scores are in TMEM before its probability group is free.
+        if (ok) ok = issue_qk();
+        if (ok && n_tiles > 1) ok = issue_qk();
+        int vs = 0;
+        uint32_t vph = 0;
         for (int64_t j = 0; ok && j < n_tiles; ++j) {
-            if (j + 2 < n_tiles) {
-                ok = issue_qk(j + 2);
-                if (!ok) break;
-            }
-            const int s = static_cast<int>(j % kStages);
-            const uint32_t ph = static_cast<uint32_t>((j / kStages) & 1);
+            if (next_qk < n_tiles && !issue_qk()) break;
             const int pb = static_cast<int>(j & 1);
-            if (!wait_barrier(&sm->v_full[s], ph, sm, P.status)) { ok = false; break; }
-            if (!wait_barrier(&sm->p_full[pb], static_cast<uint32_t>((j >> 1) & 1), sm, P.status)) { ok = false; break; }
+            if (!wait1(&sm->v_full[vs], vph, sm, P.status)) break;
+            if (!wait1(&sm->p_full[pb], static_cast<uint32_t>((j >> 1) & 1), sm, P.status)) break;
             ptx::tc_fence_after_sync();
-            if (lane == 0) {
-                const uint32_t sfp = tmem + kColSfP + 4 * pb;
-                const uint32_t sfv = tmem + kColSfV + 8 * pb;
-                ptx::tmem_cp_sf(sfp, ptx::smem_desc(ptx::smem_u32(sm->sf_p[pb]), 16, 128, ptx::kLayoutNone));
-                ptx::tmem_cp_sf(sfv, ptx::smem_desc(ptx::smem_u32(sm->sf_v[s]), 16, 128, ptx::kLayoutNone));
-                const uint32_t p_addr = ptx::smem_u32(sm->p[pb]);
-                const uint32_t v_addr = ptx::smem_u32(sm->v[s]);
-#pragma unroll
-                for (uint32_t kk = 0; kk < 2; ++kk) {
-                    const uint32_t id = kk * 2;
-                    ptx::mma_mxf4(tmem + kColO, ptx::smem_desc(p_addr + 32 * kk, 16, 512, ptx::kLayoutSw64),
-                                  ptx::smem_desc(v_addr + 32 * kk, 16, 512, ptx::kLayoutSw64), ptx::mxf4_idesc(144, id),
-                                  sfp | (id << 30), sfv | (id << 30), (j > 0 || kk > 0) ? 1u : 0u);
-                }
-                ptx::mma_commit(&sm->v_empty[s]);
-                ptx::mma_commit(&sm->p_empty[pb]);
-            }
-            __syncwarp();
+            const uint32_t sfp = tmem + kColSfP + 4 * pb;
+            const uint32_t sfv = tmem + kColSfV + 8 * pb;
+            ptx::tmem_cp_sf(sfp, d_sf + (ptx::smem_u32(sm->sf_p[pb]) >> 4));
+            ptx::tmem_cp_sf(sfv, d_sf + (ptx::smem_u32(sm->sf_v[vs]) >> 4));
+            const uint64_t dp0 = d_sw64 + (ptx::smem_u32(sm->p[pb]) >> 4);
+            const uint64_t dv0 = d_sw64 + (ptx::smem_u32(sm->v[vs]) >> 4);
+            ptx::mma_mxf4(tmem + kColO, dp0, dv0, idesc_pv0, sfp, sfv, j > 0 ? 1u : 0u);
+            ptx::mma_mxf4(tmem + kColO, dp0 + 2, dv0 + 2, idesc_pv1, sfp | (2u << 30), sfv | (2u << 30), 1u);
+            ptx::mma_commit(&sm->v_empty[vs]);
+            ptx::mma_commit(&sm->p_empty[pb]);
+            if (j + 1 == n_tiles) ptx::mma_commit(&sm->o_done);
+            if (++vs == kStages) { vs = 0; vph ^= 1u; }
         }
     }
     } else {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+    const int quarter = warp & 3;                       // TMEM lane quarter this warp may touch
+    const int group = (warp - 4) >> 2;                  // group 0 takes the even KV tiles, group 1 the odd ones
+    const uint32_t row = quarter * 32 + lane;           // row inside the query tile: one thread owns one row
+    const int64_t grow = q0 + row;                      // global query row
+    const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
     if (run) {
         // =============================== probability generation ===============================
-        const int quarter = warp & 3;                       // TMEM lane quarter this warp may touch
-        const int half = (warp - 4) >> 2;                   // which 64 keys of the tile
-        const uint32_t row = quarter * 32 + lane;           // row inside the query tile
-        const int64_t grow = q0 + row;                      // global query row
-        const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
         const ProducerConsts K = P.K;
         int64_t limit = P.causal ? grow + shift : P.Sk - 1; // last visible key of this row
         if (limit > P.Sk - 1) limit = P.Sk - 1;
@@ -392,130 +391,119 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const int64_t drow = grow - P.dbg.q_begin;
         const int64_t nblk_all = (P.Sk + 31) / 32;
         const int64_t ntile_all = (P.Sk + kTile - 1) / kTile;
-
-        float m_raw = -INFINITY;
-        float m_s = -INFINITY;
         bool ok = true;
 
-        // Scores of tile t: TMEM -> registers (this thread's 64 keys), masked, with the two block maxima;
-        // the half-row maximum is published for the partner thread that owns the other 64 keys of the row.
-        auto fetch = [&](int64_t t, float (&r)[64], float (&bmax)[2]) -> bool {
-            const int sb = static_cast<int>(t & 1);
-            const uint32_t ph2 = static_cast<uint32_t>((t >> 1) & 1);
-            if (!wait_barrier(&sm->s_full[sb], ph2, sm, P.status)) return false;
+        for (int64_t j = group; j < n_tiles; j += 2) {
+            const int sb = group;                                         // S, P and exchange buffers belong to the group
+            const uint32_t ph2 = static_cast<uint32_t>((j >> 1) & 1);
+
+            // ---- scores of tile j: TMEM -> registers (Algorithm 2, step 1 happened on the tensor core)
+            if (!wait_all(&sm->s_full[sb], ph2, sm, P.status)) { ok = false; break; }
             ptx::tc_fence_after_sync();
-            uint32_t sr[64];
-            const uint32_t s_addr = tmem + lane_base + kColS + 128 * sb + 64 * half;
-            ptx::tmem_ld32<0>(s_addr, sr);
-            ptx::tmem_ld32<32>(s_addr + 32, sr);
-            ptx::tmem_wait_ld();
-            ptx::tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&sm->s_empty[sb]);
-            const int64_t key0 = t * kTile + 64 * half;
-            if (key0 + 63 > limit) {
+            float r[128];
+            {
+                uint32_t sr[128];
+                const uint32_t s_addr = tmem + lane_base + kColS + 128 * sb;
+                ptx::tmem_ld32<0>(s_addr, sr);
+                ptx::tmem_ld32<32>(s_addr + 32, sr);
+                ptx::tmem_ld32<64>(s_addr + 64, sr);
+                ptx::tmem_ld32<96>(s_addr + 96, sr);
+                ptx::tmem_wait_ld();
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&sm->s_empty[sb]);
+                const int64_t key0 = j * kTile;
+                if (key0 + 127 > limit) {
 #pragma unroll
-                for (int i = 0; i < 64; ++i) r[i] = key0 + i > limit ? -INFINITY : __uint_as_float(sr[i]);
-            } else {
+                    for (int i = 0; i < 128; ++i) r[i] = key0 + i > limit ? -INFINITY : __uint_as_float(sr[i]);
+                } else {
 #pragma unroll
-                for (int i = 0; i < 64; ++i) r[i] = __uint_as_float(sr[i]);
+                    for (int i = 0; i < 128; ++i) r[i] = __uint_as_float(sr[i]);
+                }
             }
-            bmax[0] = block_max32(&r[0]);
-            bmax[1] = block_max32(&r[32]);
-            sm->xchg[sb][half][row] = fmaxf(bmax[0], bmax[1]);
+            float bmax[4];
+#pragma unroll
+            for (int g = 0; g < 4; ++g) bmax[g] = block_max32(&r[32 * g]);
+
+            // ---- running row maximum (Eq. rowmax-update): handed over from the group that owns tile j-1
+            float m_prev = -INFINITY;
+            if (j > 0) {
+                if (!wait_all(&sm->x_bar[sb ^ 1][quarter], static_cast<uint32_t>(((j - 1) >> 1) & 1), sm, P.status)) { ok = false; break; }
+                m_prev = sm->runmax[sb ^ 1][row];
+            }
+            const float m_new = fmaxf(fmaxf(m_prev, bmax[0]), max3(bmax[1], bmax[2], bmax[3]));
+            sm->runmax[sb][row] = m_new;
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&sm->x_bar[sb][quarter]);
-            return true;
-        };
+            const float m_s_prev = __fmul_rn(K.sigma, m_prev);
+            const float m_s = __fmul_rn(K.sigma, m_new);
+            const bool grew = m_new > m_prev && m_prev != -INFINITY;      // history exists and must be rescaled
+            const float alpha = grew ? ex2_approx(__fmul_rn(__fsub_rn(m_s_prev, m_s), K.LOG2E)) : 1.0f;
 
-        // One KV tile (Algorithm 2, steps 2-13 for this thread's half row); `nxt` is filled for tile j+1 first so
-        // that its maximum exchange overlaps this tile's code generation.
-        auto body = [&](int64_t j, float (&cur)[64], float (&cmax)[2], float (&nxt)[64], float (&nmax)[2]) -> bool {
-            const int sb = static_cast<int>(j & 1);
-            const uint32_t ph2 = static_cast<uint32_t>((j >> 1) & 1);
-            if (j + 1 < n_tiles && !fetch(j + 1, nxt, nmax)) return false;
-
-            // running row maximum (Eq. rowmax-update) with the partner's half
-            if (!wait_barrier(&sm->x_bar[sb][quarter], ph2, sm, P.status)) return false;
-            const float other = sm->xchg[sb][half ^ 1][row];
-            const float m_new = fmaxf(m_raw, max3(cmax[0], cmax[1], other));
-            const float m_s_new = __fmul_rn(K.sigma, m_new);
-            const bool grew = m_new > m_raw && m_raw != -INFINITY;   // history exists and must be rescaled
-            const float alpha = grew ? ex2_approx(__fmul_rn(__fsub_rn(m_s, m_s_new), K.LOG2E)) : 1.0f;
-            m_raw = m_new;
-            m_s = m_s_new;
-
-            // P buffer sb free?  (P~V of tile j-2 finished)
-            if (!wait_barrier(&sm->p_empty[sb], ph2 ^ 1u, sm, P.status)) return false;
-            const int64_t key0 = j * kTile + 64 * half;
-            uint32_t bytes[2];
+            // ---- probability operand (Algorithm 1 per block): codes and scales straight into the MMA operand
+            if (!wait_all(&sm->p_empty[sb], ph2 ^ 1u, sm, P.status)) { ok = false; break; }   // P~V of tile j-2 finished
+            uint32_t sfword = 0;
 #pragma unroll
-            for (int g = 0; g < 2; ++g) {
+            for (int g = 0; g < 4; ++g) {
                 uint4 codes;
-                produce32<PRODUCER, FIX8>(&cur[g * 32], cmax[g], m_s, K, codes, bytes[g]);
-                if (m_new == -INFINITY) { codes = make_uint4(0, 0, 0, 0); bytes[g] = 0; }
-                *reinterpret_cast<uint4*>(sm->p[sb] + p_swizzled_offset(row, 2 * half + g)) = codes;
+                uint32_t byte;
+                produce32<PRODUCER, FIX8>(&r[g * 32], bmax[g], m_s, K, codes, byte);
+                if (m_new == -INFINITY) { codes = make_uint4(0, 0, 0, 0); byte = 0; }
+                *reinterpret_cast<uint4*>(sm->p[sb] + p_swizzled_offset(row, g)) = codes;
+                sfword |= byte << (8 * g);
                 if (DEBUG && dbg_row) {
-                    const int64_t blk = (key0 + 32 * g) / 32;
+                    const int64_t blk = j * 4 + g;
                     if (blk < nblk_all) {
                         if (P.dbg.codes) *reinterpret_cast<uint4*>(P.dbg.codes + (drow * nblk_all + blk) * 16) = codes;
-                        if (P.dbg.scales) P.dbg.scales[drow * nblk_all + blk] = static_cast<uint8_t>(bytes[g]);
+                        if (P.dbg.scales) P.dbg.scales[drow * nblk_all + blk] = static_cast<uint8_t>(byte);
                     }
                 }
             }
-            *reinterpret_cast<uint16_t*>(sm->sf_p[sb] + (row & 31u) * 16u + (row >> 5) * 4u + 2 * half) =
-                static_cast<uint16_t>(bytes[0] | (bytes[1] << 8));
+            *reinterpret_cast<uint32_t*>(sm->sf_p[sb] + (row & 31u) * 16u + (row >> 5) * 4u) = sfword;
             if (DEBUG && dbg_row) {
                 if (P.dbg.raw_scores) {
-                    for (int i = 0; i < 64; ++i)
-                        if (key0 + i < P.Sk) P.dbg.raw_scores[drow * P.Sk + key0 + i] = cur[i];
+                    for (int i = 0; i < 128; ++i)
+                        if (j * kTile + i < P.Sk) P.dbg.raw_scores[drow * P.Sk + j * kTile + i] = r[i];
                 }
-                if (P.dbg.row_max && half == 0) P.dbg.row_max[drow * ntile_all + j] = m_s;
+                if (P.dbg.row_max) P.dbg.row_max[drow * ntile_all + j] = m_s;
             }
 
-            // historical rescaling (Eq. alpha): O rows and the denominator column in TMEM
+            // ---- historical rescaling (Eq. alpha): O rows and the denominator column in TMEM
             if (j > 0 && __any_sync(0xffffffffu, grew)) {
-                const int pv = static_cast<int>((j - 1) & 1);
-                if (!wait_barrier(&sm->p_empty[pv], static_cast<uint32_t>(((j - 1) >> 1) & 1), sm, P.status)) return false;
+                if (!wait_all(&sm->p_empty[sb ^ 1], static_cast<uint32_t>(((j - 1) >> 1) & 1), sm, P.status)) { ok = false; break; }
                 ptx::tc_fence_after_sync();
+                const uint32_t o_addr = tmem + lane_base + kColO;
                 uint32_t o[64];
-                const uint32_t o_addr = tmem + lane_base + kColO + 64 * half;
-                ptx::tmem_ld32<0>(o_addr, o);
-                ptx::tmem_ld32<32>(o_addr + 32, o);
-                uint32_t lcol = 0;
-                if (half == 1) lcol = ptx::tmem_ld1(tmem + lane_base + kColO + 128);
-                ptx::tmem_wait_ld();
 #pragma unroll
-                for (int i = 0; i < 64; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                ptx::tmem_st32<0>(o_addr, o);
-                ptx::tmem_st32<32>(o_addr + 32, o);
-                if (half == 1) ptx::tmem_st1(tmem + lane_base + kColO + 128, __float_as_uint(__uint_as_float(lcol) * alpha));
+                for (int c = 0; c < 2; ++c) {
+                    ptx::tmem_ld32<0>(o_addr + 64 * c, o);
+                    ptx::tmem_ld32<32>(o_addr + 64 * c + 32, o);
+                    ptx::tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 64; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                    ptx::tmem_st32<0>(o_addr + 64 * c, o);
+                    ptx::tmem_st32<32>(o_addr + 64 * c + 32, o);
+                    ptx::tmem_wait_st();   // the stores read o[] asynchronously: not before this may o[] be reused
+                }
+                const uint32_t lcol = ptx::tmem_ld1(o_addr + 128);
+                ptx::tmem_wait_ld();
+                ptx::tmem_st1(o_addr + 128, __float_as_uint(__uint_as_float(lcol) * alpha));
                 ptx::tmem_wait_st();
             }
             ptx::fence_proxy_async_smem();
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&sm->p_full[sb]);
-            return true;
-        };
+        }
 
-        {
-            float ra[64], rb[64], ma[2], mb[2];
-            ok = fetch(0, ra, ma);
-            for (int64_t j = 0; ok && j < n_tiles; j += 2) {
-                ok = body(j, ra, ma, rb, mb);
-                if (ok && j + 1 < n_tiles) ok = body(j + 1, rb, mb, ra, ma);
-            }
-        }
-        // ---- final normalisation O = A / l
-        if (ok) {
-            const int64_t jl = n_tiles - 1;
-            ok = wait_barrier(&sm->p_empty[jl & 1], static_cast<uint32_t>((jl >> 1) & 1), sm, P.status);
-        }
+        // ---- final normalisation O = A / l: each group writes 64 of the 128 channels
+        // (a barrier of its own: a group that skipped a phase of the other group's p_empty could not tell
+        // an old completion from the last one by parity)
+        if (ok) ok = wait_all(&sm->o_done, 0, sm, P.status);
         if (ok) {
             ptx::tc_fence_after_sync();
             uint32_t o[64];
-            const uint32_t o_addr = tmem + lane_base + kColO + 64 * half;
+            const uint32_t o_addr = tmem + lane_base + kColO + 64 * group;
             ptx::tmem_ld32<0>(o_addr, o);
             ptx::tmem_ld32<32>(o_addr + 32, o);
             const uint32_t lcol = ptx::tmem_ld1(tmem + lane_base + kColO + 128);
@@ -523,7 +511,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             if (grow < P.Sq) {
                 const float l = __uint_as_float(lcol);
                 const float inv = l > 0.0f ? 1.0f / l : 0.0f;
-                float4* dst = reinterpret_cast<float4*>(P.o + ((bh * P.Sq + grow) * 128 + 64 * half));
+                float4* dst = reinterpret_cast<float4*>(P.o + ((bh * P.Sq + grow) * 128 + 64 * group));
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
                     float4 v;
@@ -537,10 +525,8 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         }
     } else if (sm->abort_flag == 0) {
         // no visible key for the whole tile: rows are zero
-        const int quarter = warp & 3, half = (warp - 4) >> 2;
-        const int64_t grow = q0 + quarter * 32 + lane;
         if (grow < P.Sq) {
-            float4* dst = reinterpret_cast<float4*>(P.o + ((bh * P.Sq + grow) * 128 + 64 * half));
+            float4* dst = reinterpret_cast<float4*>(P.o + ((bh * P.Sq + grow) * 128 + 64 * group));
             for (int i = 0; i < 16; ++i) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
     }
@@ -704,6 +690,13 @@ efq_status_t attention_impl(const void* q, const void* k, const void* v, float* 
 
 }  // namespace
 }  // namespace efq
+
+#ifdef EFQ_TIMELINE
+extern "C" int efq_dev_set_timeline(long long* buf)
+{
+    return static_cast<int>(cudaMemcpyToSymbol(efq::g_timeline, &buf, sizeof(buf)));
+}
+#endif
 
 extern "C" size_t efq_attention_workspace_bytes(int B, int Hq, int Hkv, int64_t Sq, int64_t Sk, int d)
 {
