@@ -4,9 +4,9 @@
 // One CTA owns one 128-row query tile of one (batch, head) and walks the KV tiles of width 128:
 //   warp 0      TMA producer: Q tile once, then K_j / V^T_j code tiles (SW64 layout) and their
 //               512-byte scale tiles through 4-stage mbarrier rings
-//   warp 1      MMA issuer (one elected thread): scale tiles smem -> TMEM (tcgen05.cp), then
-//               S_j = Q^ K^_j^T  and  [dA | dl] = P~_j [V^_j | 1]  as kind::mxf4 block-scaled MMAs,
-//               FP32 accumulators in TMEM.  The 16 "ones" rows appended to V^T give the denominator
+//   warps 1, 2  MMA issuers (one elected lane each): scale tiles smem -> TMEM (tcgen05.cp), then warp 1
+//               S_j = Q^ K^_j^T  and warp 2  [dA | dl] = P~_j [V^_j | 1]  as kind::mxf4 block-scaled MMAs,
+//               FP32 accumulators in TMEM; S runs up to two tiles ahead of P~V.  The 16 "ones" rows appended to V^T give the denominator
 //               P~1 from the very operand that feeds the numerator.
 //   warps 4-11  probability generation, two groups of four warps: group 0 takes the even KV tiles,
 //               group 1 the odd ones, so one group's latency-bound steps (TMEM load, hand-over of the
@@ -300,6 +300,8 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         int s = 0;
         uint32_t ph = 0;
         for (int64_t j = 0; j < n_tiles; ++j) {
+            // Stage barriers of their own: a waiter on a barrier that other roles may complete twice before it
+            // looks (S runs ahead) could not tell which completion it sees by parity.
             if (!wait1(&sm->k_empty[s], ph ^ 1u, sm, P.status)) break;
             ptx::mbar_arrive_expect_tx(&sm->k_full[s], kTileBytes + kSfBytes);
             ptx::tma_load_2d(sm->k[s], &map_k, 0, static_cast<int>(kvh * P.Sk_pad + j * kTile), &sm->k_full[s]);
@@ -310,67 +312,68 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             ptx::bulk_load_1d(sm->sf_v[s], P.sf_v + (kvh * kv_tiles + j) * kSfBytes, kSfBytes, &sm->v_full[s]);
             if (++s == kStages) { s = 0; ph ^= 1u; }
         }
-    } else if (run && warp == 1 && lane == 0) {
-        // =============================== MMA issuer (one thread) ===============================
-        // Descriptors differ from tile to tile only in the start-address field (address >> 4).
+    } else if (run && warp == 1) {
+        // =============================== S = Q K^T issuer ===============================
+        // The whole warp runs the loop with warp-uniform state; one elected lane issues the tcgen05
+        // instructions.  Descriptors differ from tile to tile only in the start-address field (address >> 4).
         const uint64_t d_sw64 = ptx::smem_desc(0, 16, 512, ptx::kLayoutSw64);
         const uint64_t d_sf = ptx::smem_desc(0, 16, 128, ptx::kLayoutNone);
         const uint64_t dq0 = d_sw64 + (ptx::smem_u32(sm->q) >> 4);
-        const uint32_t idesc_qk0 = ptx::mxf4_idesc(128, 0), idesc_qk1 = ptx::mxf4_idesc(128, 2);
-        const uint32_t idesc_pv0 = ptx::mxf4_idesc(144, 0), idesc_pv1 = ptx::mxf4_idesc(144, 2);
         const uint32_t sfq = tmem + kColSfQ;
-        bool ok = wait1(&sm->q_full, 0, sm, P.status);
+        bool ok = wait_all(&sm->q_full, 0, sm, P.status);
         ptx::tc_fence_after_sync();
-        if (ok) {
-            ptx::tmem_cp_sf(sfq, d_sf + (ptx::smem_u32(sm->sf_q) >> 4));
+        if (ok && ptx::elect_one()) ptx::tmem_cp_sf(sfq, d_sf + (ptx::smem_u32(sm->sf_q) >> 4));
+        int ks = 0;
+        uint32_t kph = 0;
+        for (int64_t t = 0; ok && t < n_tiles; ++t) {
+            const int sb = static_cast<int>(t & 1);
+            if (!wait_all(&sm->k_full[ks], kph, sm, P.status)) break;
+            if (!wait_all(&sm->s_empty[sb], static_cast<uint32_t>((t >> 1) & 1) ^ 1u, sm, P.status)) break;
+            ptx::tc_fence_after_sync();
+            if (ptx::elect_one()) {
+                const uint32_t sfk = tmem + kColSfK + 4 * sb;
+                ptx::tmem_cp_sf(sfk, d_sf + (ptx::smem_u32(sm->sf_k[ks]) >> 4));
+                const uint64_t dk0 = d_sw64 + (ptx::smem_u32(sm->k[ks]) >> 4);
+                const uint32_t d_s = tmem + kColS + 128 * sb;
+                ptx::mma_mxf4(d_s, dq0, dk0, ptx::mxf4_idesc(128, 0), sfq, sfk, 0u);
+                ptx::mma_mxf4(d_s, dq0 + 2, dk0 + 2, ptx::mxf4_idesc(128, 2), sfq | (2u << 30), sfk | (2u << 30), 1u);
+                ptx::mma_commit(&sm->s_full[sb]);
+                ptx::mma_commit(&sm->k_empty[ks]);
+            }
+            __syncwarp();
+            if (++ks == kStages) { ks = 0; kph ^= 1u; }
+        }
+    } else if (run && warp == 2) {
+        // =============================== [dA | dl] = P~ [V | 1] issuer ===============================
+        const uint64_t d_sw64 = ptx::smem_desc(0, 16, 512, ptx::kLayoutSw64);
+        const uint64_t d_sf = ptx::smem_desc(0, 16, 128, ptx::kLayoutNone);
+        if (ptx::elect_one()) {
             const uint64_t d1 = d_sf + (ptx::smem_u32(sm->sf_ones) >> 4);
             ptx::tmem_cp_sf(tmem + kColSfV + 4, d1);
             ptx::tmem_cp_sf(tmem + kColSfV + 12, d1);
         }
-        int ks = 0;                 // K ring position of the next QK to issue
-        uint32_t kph = 0;
-        int64_t next_qk = 0;
-        // QK_t: S[t&1] = Q K_t^T
-        auto issue_qk = [&]() -> bool {
-            const int64_t t = next_qk;
-            const int sb = static_cast<int>(t & 1);
-            if (!wait1(&sm->k_full[ks], kph, sm, P.status)) return false;
-            if (!wait1(&sm->s_empty[sb], static_cast<uint32_t>((t >> 1) & 1) ^ 1u, sm, P.status)) return false;
-            ptx::tc_fence_after_sync();
-            const uint32_t sfk = tmem + kColSfK + 4 * sb;
-            ptx::tmem_cp_sf(sfk, d_sf + (ptx::smem_u32(sm->sf_k[ks]) >> 4));
-            const uint64_t dk0 = d_sw64 + (ptx::smem_u32(sm->k[ks]) >> 4);
-            const uint32_t d_s = tmem + kColS + 128 * sb;
-            ptx::mma_mxf4(d_s, dq0, dk0, idesc_qk0, sfq, sfk, 0u);
-            ptx::mma_mxf4(d_s, dq0 + 2, dk0 + 2, idesc_qk1, sfq | (2u << 30), sfk | (2u << 30), 1u);
-            ptx::mma_commit(&sm->k_empty[ks]);
-            ptx::mma_commit(&sm->s_full[sb]);
-            if (++ks == kStages) { ks = 0; kph ^= 1u; }
-            ++next_qk;
-            return true;
-        };
-        // S runs two tiles ahead of P~V so that a tile's scores are in TMEM before its probability group is free.
-        if (ok) ok = issue_qk();
-        if (ok && n_tiles > 1) ok = issue_qk();
+        __syncwarp();
         int vs = 0;
         uint32_t vph = 0;
-        for (int64_t j = 0; ok && j < n_tiles; ++j) {
-            if (next_qk < n_tiles && !issue_qk()) break;
+        for (int64_t j = 0; j < n_tiles; ++j) {
             const int pb = static_cast<int>(j & 1);
-            if (!wait1(&sm->v_full[vs], vph, sm, P.status)) break;
-            if (!wait1(&sm->p_full[pb], static_cast<uint32_t>((j >> 1) & 1), sm, P.status)) break;
+            if (!wait_all(&sm->v_full[vs], vph, sm, P.status)) break;
+            if (!wait_all(&sm->p_full[pb], static_cast<uint32_t>((j >> 1) & 1), sm, P.status)) break;
             ptx::tc_fence_after_sync();
-            const uint32_t sfp = tmem + kColSfP + 4 * pb;
-            const uint32_t sfv = tmem + kColSfV + 8 * pb;
-            ptx::tmem_cp_sf(sfp, d_sf + (ptx::smem_u32(sm->sf_p[pb]) >> 4));
-            ptx::tmem_cp_sf(sfv, d_sf + (ptx::smem_u32(sm->sf_v[vs]) >> 4));
-            const uint64_t dp0 = d_sw64 + (ptx::smem_u32(sm->p[pb]) >> 4);
-            const uint64_t dv0 = d_sw64 + (ptx::smem_u32(sm->v[vs]) >> 4);
-            ptx::mma_mxf4(tmem + kColO, dp0, dv0, idesc_pv0, sfp, sfv, j > 0 ? 1u : 0u);
-            ptx::mma_mxf4(tmem + kColO, dp0 + 2, dv0 + 2, idesc_pv1, sfp | (2u << 30), sfv | (2u << 30), 1u);
-            ptx::mma_commit(&sm->v_empty[vs]);
-            ptx::mma_commit(&sm->p_empty[pb]);
-            if (j + 1 == n_tiles) ptx::mma_commit(&sm->o_done);
+            if (ptx::elect_one()) {
+                const uint32_t sfp = tmem + kColSfP + 4 * pb;
+                const uint32_t sfv = tmem + kColSfV + 8 * pb;
+                ptx::tmem_cp_sf(sfp, d_sf + (ptx::smem_u32(sm->sf_p[pb]) >> 4));
+                ptx::tmem_cp_sf(sfv, d_sf + (ptx::smem_u32(sm->sf_v[vs]) >> 4));
+                const uint64_t dp0 = d_sw64 + (ptx::smem_u32(sm->p[pb]) >> 4);
+                const uint64_t dv0 = d_sw64 + (ptx::smem_u32(sm->v[vs]) >> 4);
+                ptx::mma_mxf4(tmem + kColO, dp0, dv0, ptx::mxf4_idesc(144, 0), sfp, sfv, j > 0 ? 1u : 0u);
+                ptx::mma_mxf4(tmem + kColO, dp0 + 2, dv0 + 2, ptx::mxf4_idesc(144, 2), sfp | (2u << 30), sfv | (2u << 30), 1u);
+                ptx::mma_commit(&sm->p_empty[pb]);
+                ptx::mma_commit(&sm->v_empty[vs]);
+                if (j + 1 == n_tiles) ptx::mma_commit(&sm->o_done);
+            }
+            __syncwarp();
             if (++vs == kStages) { vs = 0; vph ^= 1u; }
         }
     }
