@@ -114,11 +114,13 @@ __device__ __forceinline__ bool wait1(uint64_t* bar, uint32_t parity, Smem* sm, 
         }
     }
 }
-// The same wait executed by all lanes of a warp; the verdict is made warp-uniform.
+// The same wait executed by all lanes of a warp.  All lanes poll the same barrier; only the rare timeout path
+// can split a warp, so the verdict is made warp-uniform there and nowhere else.
 __device__ __forceinline__ bool wait_all(uint64_t* bar, uint32_t parity, Smem* sm, uint32_t* status)
 {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
     const bool ok = wait1(bar, parity, sm, status);
-    return __all_sync(0xffffffffu, ok);
+    return __all_sync(__activemask(), ok);
 }
 
 __device__ __forceinline__ uint32_t p_swizzled_offset(uint32_t row, uint32_t chunk)
@@ -191,7 +193,7 @@ __device__ __forceinline__ void produce32(const float* r, float rmax, float m_s,
             asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(a2));
             uint32_t word = __byte_perm(lo, hi, 0x5410);
             if (FIX8) word -= (word >> 3) & 0x11111111u;
-            w[q] = s.live ? word : 0u;
+            w[q] = word;   // a block without a finite score has w = 0 everywhere (sat(-inf) and sat(NaN) are 0)
         }
     } else {
         float p[32];
@@ -404,6 +406,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             if (!wait_all(&sm->s_full[sb], ph2, sm, P.status)) { ok = false; break; }
             ptx::tc_fence_after_sync();
             float r[128];
+            float bmax[4];
             {
                 uint32_t sr[128];
                 const uint32_t s_addr = tmem + lane_base + kColS + 128 * sb;
@@ -424,7 +427,6 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                     for (int i = 0; i < 128; ++i) r[i] = __uint_as_float(sr[i]);
                 }
             }
-            float bmax[4];
 #pragma unroll
             for (int g = 0; g < 4; ++g) bmax[g] = block_max32(&r[32 * g]);
 
@@ -451,7 +453,6 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 uint4 codes;
                 uint32_t byte;
                 produce32<PRODUCER, FIX8>(&r[g * 32], bmax[g], m_s, K, codes, byte);
-                if (m_new == -INFINITY) { codes = make_uint4(0, 0, 0, 0); byte = 0; }
                 *reinterpret_cast<uint4*>(sm->p[sb] + p_swizzled_offset(row, g)) = codes;
                 sfword |= byte << (8 * g);
                 if (DEBUG && dbg_row) {
