@@ -39,7 +39,8 @@ typedef enum {
     EFQ_ERR_WORKSPACE = 4,      /* workspace pointer null or smaller than efq_attention_workspace_bytes() */
     EFQ_ERR_ARCH = 5,           /* current device is not compute capability 10.x */
     EFQ_ERR_CUDA = 6,           /* a CUDA runtime/driver call failed (launch, copy, descriptor encode) */
-    EFQ_ERR_DEVICE_TIMEOUT = 7  /* a bounded device-side wait expired; the output is invalid */
+    EFQ_ERR_DEVICE_TIMEOUT = 7, /* a bounded device-side wait expired; the output is invalid */
+    EFQ_ERR_STATIC_LIMIT = 8    /* efq_attention_fwd_static: the problem needs more than EFQ_STATIC_SCRATCH_BYTES */
 } efq_status_t;
 
 /* Parameters of the affine code rule c = clip_[0,7](floor((z - tau) h) + 1)
@@ -146,6 +147,35 @@ efq_status_t efq_attention_fwd_host(const void* q_host, const void* k_host, cons
                                     int64_t Sq, int64_t Sk, int d, int causal, float softmax_scale, int producer,
                                     const efq_params_t* params, void* workspace, size_t workspace_bytes,
                                     void* stream);
+
+/* Built-in scratch of efq_attention_fwd_static, in bytes (4 MiB).  Enough for, e.g., one head of 8192 tokens or
+ * 8 query / 2 KV heads of 2048 tokens; efq_attention_workspace_bytes() gives the need of a shape. */
+#define EFQ_STATIC_SCRATCH_BYTES (4u << 20)
+
+/* efq_attention_fwd for callers that have no device memory to hand over as workspace.  (The paper has no
+ * counterpart: this is a packaging variant of efq_attention_fwd, same arithmetic, same results.)
+ *
+ * Who needs it: code that runs where device allocation is off the table - a serving loop that must not call
+ * cudaMalloc after start-up because the call synchronises the device and can fail once the memory pool is
+ * fully handed out, or a plug-in living inside a host application that owns all device memory and gives
+ * none of it to the plug-in.  Such a caller still owns q, k, v and o, but cannot produce the MXFP4 workspace.
+ *
+ * What it does instead: the MXFP4 copies of Q, K, V, their scale tiles and the status word go into a fixed
+ * array of EFQ_STATIC_SCRATCH_BYTES that is part of the library image (so every device that loads the
+ * library holds these bytes until the process exits).  The call allocates and frees nothing.
+ *   - Shapes whose workspace would exceed the array are refused with EFQ_ERR_STATIC_LIMIT; nothing is
+ *     launched.  Other argument rules and error codes are those of efq_attention_fwd (no debug dump).
+ *   - The first call on each device looks up the array's device address (a host-side step, done with that
+ *     device current, protected by a lock).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps whatever the previous call left; each call
+ *     rewrites every byte it later reads and clears the status word first.  Two calls whose GPU work
+ *     overlaps (different streams, or one stream from several threads without ordering) race on the array:
+ *     serialise them.  The status word sits in the same array and this entry point has no poll call: a
+ *     caller that must detect a device-side timeout uses efq_attention_fwd with a workspace of its own
+ *     and efq_poll_status. */
+efq_status_t efq_attention_fwd_static(const void* q, const void* k, const void* v, float* o, int B, int Hq, int Hkv,
+                                      int64_t Sq, int64_t Sk, int d, int causal, float softmax_scale,
+                                      const efq_params_t* params, void* stream);
 
 /* Synchronises `stream` and returns the device-side status word of the last forward that
  * used `workspace` (EFQ_OK, or EFQ_ERR_DEVICE_TIMEOUT if a bounded wait expired), or

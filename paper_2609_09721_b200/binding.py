@@ -17,12 +17,13 @@ LIB_PATH = os.path.join(_HERE, "libefq_b200.so")
 
 EFQ_OK = 0
 STATUS_NAMES = ["EFQ_OK", "EFQ_ERR_INVALID_ARG", "EFQ_ERR_UNSUPPORTED", "EFQ_ERR_ALIGNMENT", "EFQ_ERR_WORKSPACE",
-                "EFQ_ERR_ARCH", "EFQ_ERR_CUDA", "EFQ_ERR_DEVICE_TIMEOUT"]
+                "EFQ_ERR_ARCH", "EFQ_ERR_CUDA", "EFQ_ERR_DEVICE_TIMEOUT", "EFQ_ERR_STATIC_LIMIT"]
+STATIC_SCRATCH_BYTES = 4 << 20
 
 # every symbol include/efq.h declares
 EXPORTS = ["efq_probgen", "exp_then_quantize_probgen", "efq_attention_workspace_bytes", "efq_attention_fwd",
            "exp_then_quantize_attention_fwd", "efq_quantize_qkv", "efq_attention_fwd_quantized",
-           "efq_attention_fwd_host", "efq_poll_status",
+           "efq_attention_fwd_host", "efq_attention_fwd_static", "efq_poll_status",
            "efq_fp4_mma_peak_probe", "efq_status_string", "efq_version"]
 
 
@@ -74,6 +75,9 @@ def lib() -> C.CDLL:
         L.efq_attention_fwd_host.restype = i32
         L.efq_attention_fwd_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i64, i64, i32, i32, f32,
                                              i32, C.POINTER(EfqParams), vp, C.c_size_t, vp]
+        L.efq_attention_fwd_static.restype = i32
+        L.efq_attention_fwd_static.argtypes = [vp, vp, vp, vp, i32, i32, i32, i64, i64, i32, i32, f32,
+                                               C.POINTER(EfqParams), vp]
         L.efq_poll_status.restype = i32
         L.efq_poll_status.argtypes = [vp, vp]
         L.efq_fp4_mma_peak_probe.restype = i32
@@ -253,6 +257,26 @@ def efq_attention_fwd_host(q_host, k_host, v_host, o_host, q_dev, k_dev, v_dev, 
                                       workspace.numel(), _stream(stream))
     _check(st, "efq_attention_fwd_host")
     return o_host
+
+
+def efq_attention_fwd_static(q, k, v, causal: bool = False, softmax_scale: float = 0.0, params=None, o=None,
+                             stream=None):
+    """efq_attention_fwd for callers that cannot hand over a workspace: the scratch is a fixed array inside
+    the library (STATIC_SCRATCH_BYTES); larger problems raise EfqError with EFQ_ERR_STATIC_LIMIT.  The output
+    tensor is still the caller's: pass ``o`` to keep this call free of allocations."""
+    assert q.is_cuda and q.dtype == torch.bfloat16 and q.is_contiguous() and q.dim() == 4
+    assert k.is_cuda and k.dtype == torch.bfloat16 and k.is_contiguous() and k.shape == v.shape
+    assert v.is_cuda and v.dtype == torch.bfloat16 and v.is_contiguous()
+    B, Hq, Sq, d = q.shape
+    _, Hkv, Sk, _ = k.shape
+    if o is None:
+        o = torch.empty((B, Hq, Sq, d), dtype=torch.float32, device=q.device)
+    p = _params(params)
+    st = lib().efq_attention_fwd_static(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, Hq, Hkv, Sq, Sk, d,
+                                        int(bool(causal)), float(softmax_scale),
+                                        C.byref(p) if p is not None else None, _stream(stream))
+    _check(st, "efq_attention_fwd_static")
+    return o
 
 
 def efq_poll_status(workspace, stream=None) -> int:

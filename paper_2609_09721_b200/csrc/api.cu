@@ -12,6 +12,7 @@ extern "C" const char* efq_status_string(efq_status_t status)
         case EFQ_ERR_ARCH: return "device is not compute capability 10.x";
         case EFQ_ERR_CUDA: return "CUDA call failed";
         case EFQ_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+        case EFQ_ERR_STATIC_LIMIT: return "problem exceeds the built-in scratch of the no-allocation entry point";
     }
     return "unknown status";
 }

@@ -24,6 +24,8 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <mutex>
+
 #include "efq_common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -798,4 +800,54 @@ extern "C" efq_status_t efq_poll_status(void* workspace, void* stream)
     if (cudaMemcpyAsync(&word, workspace, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return EFQ_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return EFQ_ERR_CUDA;
     return word == 0 ? EFQ_OK : (word == EFQ_ERR_DEVICE_TIMEOUT ? EFQ_ERR_DEVICE_TIMEOUT : EFQ_ERR_CUDA);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Forward without a caller-supplied workspace
+// ------------------------------------------------------------------------------------------------
+// Scratch for efq_attention_fwd_static: lives in the library image, one copy per device that loads it.
+static __device__ __align__(256) uint8_t g_static_scratch[EFQ_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_ptr[kMaxDevices] = {};   // device address of g_static_scratch, per device ordinal
+
+// The array's name is only a host-side handle; kernels need its device address, which differs per device.
+// Looked up once per device with that device current.
+efq_status_t static_scratch_for_current_device(void** out)
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return EFQ_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return EFQ_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return EFQ_ERR_CUDA;
+        g_static_ptr[dev] = p;
+    }
+    *out = g_static_ptr[dev];
+    return EFQ_OK;
+}
+
+}  // namespace
+
+extern "C" efq_status_t efq_attention_fwd_static(const void* q, const void* k, const void* v, float* o, int B, int Hq,
+                                                 int Hkv, int64_t Sq, int64_t Sk, int d, int causal,
+                                                 float softmax_scale, const efq_params_t* params, void* stream)
+{
+    float tau, h;
+    efq_status_t st;
+    if (!read_params(params, tau, h, st)) return st;
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0) return EFQ_ERR_INVALID_ARG;
+    if (d != 128) return EFQ_ERR_UNSUPPORTED;
+    const size_t need = efq_attention_workspace_bytes(B, Hq, Hkv, Sq, Sk, d);
+    if (need == 0) return EFQ_ERR_UNSUPPORTED;
+    if (need > EFQ_STATIC_SCRATCH_BYTES) return EFQ_ERR_STATIC_LIMIT;
+    void* scratch = nullptr;
+    st = static_scratch_for_current_device(&scratch);
+    if (st != EFQ_OK) return st;
+    return efq::attention_impl(q, k, v, o, B, Hq, Hkv, Sq, Sk, d, causal, softmax_scale, 0, tau, h, scratch,
+                               EFQ_STATIC_SCRATCH_BYTES, nullptr, static_cast<cudaStream_t>(stream), true, true);
 }
