@@ -173,6 +173,23 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def max_over_ranks(values, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks of the default process group
+    (the values themselves when no group is initialised).  Timings are reported as the slowest rank's."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.tolist()]
+
+
+def whole_job_tflops(flops_per_replica: float, ms_per_step: float, world: int) -> float:
+    """Aggregate throughput of `world` independent replicas that all finish within ms_per_step."""
+    return world * flops_per_replica / (ms_per_step * 1e-3) / 1e12
+
+
 # ------------------------------------------------------------------------------------------
 # CUDA arm
 # ------------------------------------------------------------------------------------------
@@ -236,10 +253,7 @@ def run_cuda(args):
         clocks = sampler.stop(t0, t1) if sampler else None
         ms = e0.elapsed_time(e1)
         main_ms = sum(a.elapsed_time(b) for a, b in evs) / steps
-        if world > 1:
-            t = torch.tensor([ms, main_ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms, main_ms = float(t[0]), float(t[1])
+        ms, main_ms = max_over_ranks([ms, main_ms], dev)
         return ms / steps, main_ms, clocks
 
     phys_gpu = local_rank
@@ -268,11 +282,7 @@ def run_cuda(args):
         binding.efq_attention_fwd_host(hq, hk, hv, ho, dq, dk, dv, o, case.causal, 0.0, 0, None, ws)
     e1.record(stream)
     barrier()
-    e2e_ms = e0.elapsed_time(e1) / e2e_steps
-    if world > 1:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t[0])
+    e2e_ms = max_over_ranks([e0.elapsed_time(e1) / e2e_steps], dev)[0]
     h2d = hq.numel() * 2 + hk.numel() * 2 + hv.numel() * 2
     d2h = ho.numel() * 4
 
@@ -312,7 +322,7 @@ def run_cuda(args):
 
     peaks = measured_peaks()
     flops = case.flops
-    value = world * flops / (ms_step * 1e-3) / 1e12
+    value = whole_job_tflops(flops, ms_step, world)
     main_tflops = flops / (ms_main * 1e-3) / 1e12
     fp4_peak = peaks["bf16_sustained"] * NOMINAL_FP4_OVER_BF16
     traffic = None
@@ -324,7 +334,7 @@ def run_cuda(args):
     cpu_baseline = None
     if world == 1 and not args.skip_cpu_baseline:
         q32, k32, v32 = (inputs.bf16_bits_to_f32(t) for t in (qb, kb, vb))
-        n_rows = args.oracle_rows
+        n_rows = 4 * args.oracle_rows
         cv, csec, cores = time_oracle(case, q32, k32, v32, n_rows, 3, 1)
         cpu_baseline = {"value": cv, "unit": UNIT, "cores": cores, "kind": "oracle",
                         "sample": f"3 steps of {n_rows} seeded query rows (all heads), EFQ path, {csec:.2f} s per step"}
@@ -337,7 +347,7 @@ def run_cuda(args):
                    "causal": case.causal, "kv_tile": 128, "params": "EFQ-Mean tau=-3.06 h=2.30",
                    "l2": "inputs larger than L2 (Q+K+V bf16 and fp32 O exceed 126 MB)", "parallelism": f"replicas x{world}"},
         "clocks": clocks,
-        "e2e": {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
+        "e2e": {"value": whole_job_tflops(flops, e2e_ms, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
         "gpu_launches": 4 * args.steps,
         "roofline": {"kernel": "attention_fwd_kernel<EFQ>", "bound": "tensor", "achieved": main_tflops, "peak": fp4_peak,
@@ -358,11 +368,12 @@ def run_cuda(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="qwen3_8b_16k")
-    ap.add_argument("--oracle-rows", type=int, default=512)
+    ap.add_argument("--oracle-rows", type=int, default=2048,
+                    help="query rows the oracle computes per step (reference arm); the cpu_baseline leg uses 4x")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-stage", action="store_true")
     args = ap.parse_args()
