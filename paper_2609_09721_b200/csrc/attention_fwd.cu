@@ -8,6 +8,8 @@
 //               S_j = Q^ K^_j^T  and warp 2  [dA | dl] = P~_j [V^_j | 1]  as kind::mxf4 block-scaled MMAs,
 //               FP32 accumulators in TMEM; S runs up to two tiles ahead of P~V.  The 16 "ones" rows appended to V^T give the denominator
 //               P~1 from the very operand that feeds the numerator.
+//   warps 12-15 historical rescaling: when a row's maximum grew in tile j, its accumulator row and denominator in
+//               TMEM are multiplied by alpha_j after P~V_{j-1} and before P~V_j, beside the code generation.
 //   warps 4-11  probability generation, two groups of four warps: group 0 takes the even KV tiles,
 //               group 1 the odd ones, so one group's latency-bound steps (TMEM load, hand-over of the
 //               running maximum, accumulator rescaling) overlap the other group's code generation.
@@ -16,7 +18,7 @@
 //               the swizzled shared-memory A operand, the four scale bytes as one word into the scale
 //               tile.  No FP16/FP32 probability tile exists anywhere.
 // The online recurrence is unchanged: when a row's maximum grows, the accumulator rows in TMEM
-// are rescaled by alpha = exp(m_old - m_new) before the next P~V MMA is released.
+// are rescaled by alpha = exp(m_old - m_new) before the next P~V MMA is released (warps 12-15).
 //
 // TMEM columns: S double buffer 2 x 128 | O 144 (128 channels + 16 denominator) | scale factors.
 // Every wait is bounded; on expiry the CTA records EFQ_ERR_DEVICE_TIMEOUT in the workspace status
@@ -48,7 +50,7 @@ namespace {
 
 constexpr int kTile = 128;            // query rows per CTA and keys per KV tile (Bc)
 constexpr int kStages = 4;            // K and V ring depth
-constexpr int kThreads = 384;         // 12 warps = 3 warpgroups: {TMA, MMA, 2 idle}, 2 x probability generation
+constexpr int kThreads = 512;         // 16 warps = 4 warpgroups: {TMA, QK, PV, idle}, 2 x probability generation, rescaling
 constexpr int kGroupWarps = 4;        // warps per probability group (one thread per query row)
 constexpr int kTileBytes = kTile * 64;          // 128 rows x 64 B of packed E2M1
 constexpr int kSfBytes = 512;
@@ -75,12 +77,15 @@ struct __align__(1024) Smem {
     uint8_t sf_p[2][kSfBytes];
     uint8_t sf_ones[kSfBytes];
     float runmax[2][kTile];   // running row maximum after the group's latest tile, raw score units
+    float alpha[2][kTile];    // rescale factor of the group's current tile, per row (1 where the maximum did not grow)
     uint64_t q_full;
     uint64_t k_full[kStages], k_empty[kStages];
     uint64_t v_full[kStages], v_empty[kStages];
     uint64_t s_full[2], s_empty[2];
     uint64_t p_full[2], p_empty[2];
     uint64_t x_bar[2][4];     // [group][lane quarter]: runmax of the group's latest tile is published
+    uint64_t a_bar[2][4];     // [group][lane quarter]: alpha of the group's current tile is published
+    uint64_t o_ready[2];      // accumulator rows rescaled (or found unchanged) for the tile of this parity
     uint64_t o_done;          // the last P~V of the work item has completed
     uint32_t tmem_base;
     volatile uint32_t abort_flag;
@@ -102,17 +107,21 @@ struct FwdParams {
 };
 
 // Bounded wait of one thread.  Returns false on timeout (recorded in the status word) or CTA-wide abort.
+// The polling loop is kept to the barrier test itself; the abort flag and the clock are looked at every 64th
+// round only, because every instruction a waiting warp issues is taken from the warps that compute.
 __device__ __forceinline__ bool wait1(uint64_t* bar, uint32_t parity, Smem* sm, uint32_t* status)
 {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
-    while (true) {
+    for (uint32_t spins = 1;; ++spins) {
         if (ptx::mbar_try_wait_suspend(bar, parity, 20000u)) return true;
-        if (sm->abort_flag) return false;
-        if (static_cast<uint64_t>(clock64() - t0) > kTimeoutCycles) {
-            sm->abort_flag = 1;
-            atomicExch(status, static_cast<uint32_t>(EFQ_ERR_DEVICE_TIMEOUT));
-            return false;
+        if ((spins & 63u) == 0u) {
+            if (sm->abort_flag) return false;
+            if (static_cast<uint64_t>(clock64() - t0) > kTimeoutCycles) {
+                sm->abort_flag = 1;
+                atomicExch(status, static_cast<uint32_t>(EFQ_ERR_DEVICE_TIMEOUT));
+                return false;
+            }
         }
     }
 }
@@ -273,7 +282,11 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             ptx::mbar_init(&sm->s_empty[i], kGroupWarps);
             ptx::mbar_init(&sm->p_full[i], kGroupWarps);
             ptx::mbar_init(&sm->p_empty[i], 1);
-            for (int qd = 0; qd < 4; ++qd) ptx::mbar_init(&sm->x_bar[i][qd], 1);
+            ptx::mbar_init(&sm->o_ready[i], 4);
+            for (int qd = 0; qd < 4; ++qd) {
+                ptx::mbar_init(&sm->x_bar[i][qd], 1);
+                ptx::mbar_init(&sm->a_bar[i][qd], 1);
+            }
         }
         sm->abort_flag = (*reinterpret_cast<volatile uint32_t*>(P.status) != 0u) ? 1u : 0u;
         ptx::mbar_init_fence();
@@ -363,6 +376,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             const int pb = static_cast<int>(j & 1);
             if (!wait_all(&sm->v_full[vs], vph, sm, P.status)) break;
             if (!wait_all(&sm->p_full[pb], static_cast<uint32_t>((j >> 1) & 1), sm, P.status)) break;
+            if (!wait_all(&sm->o_ready[pb], static_cast<uint32_t>((j >> 1) & 1), sm, P.status)) break;
             ptx::tc_fence_after_sync();
             if (ptx::elect_one()) {
                 const uint32_t sfp = tmem + kColSfP + 4 * pb;
@@ -381,8 +395,56 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             if (++vs == kStages) { vs = 0; vph ^= 1u; }
         }
     }
+    } else if (warp >= 12) {
+    // =============================== historical rescaling (Eq. alpha) ===============================
+    // One warp per TMEM lane quarter.  When a row's maximum grew in tile j, its accumulator row and its
+    // denominator are multiplied by alpha_j after P~V_{j-1} has landed and before P~V_j is released; this runs
+    // beside the code generation of tile j instead of inside it.
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+    const int quarter = warp & 3;
+    const uint32_t row = quarter * 32 + lane;
+    const uint32_t o_addr = tmem + (static_cast<uint32_t>(quarter * 32) << 16) + kColO;
+    if (run) {
+        for (int64_t j = 0; j < n_tiles; ++j) {
+            const int sb = static_cast<int>(j & 1);
+            // every tile, so that each phase of this barrier is seen in order
+            if (!wait_all(&sm->a_bar[sb][quarter], static_cast<uint32_t>((j >> 1) & 1), sm, P.status)) break;
+            if (j > 0) {
+                const float alpha = sm->alpha[sb][row];
+                const bool any = __any_sync(0xffffffffu, alpha != 1.0f);
+                // every tile, so that each phase of this barrier is seen in order
+                if (!wait_all(&sm->p_empty[sb ^ 1], static_cast<uint32_t>(((j - 1) >> 1) & 1), sm, P.status)) break;
+                if (any) {
+                    ptx::tc_fence_after_sync();
+                    uint32_t o[32];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        ptx::tmem_ld32<0>(o_addr + 32 * c, o);
+                        ptx::tmem_wait_ld();
+                        const uint64_t alpha2 = pack2(alpha, alpha);
+#pragma unroll
+                        for (int i = 0; i < 32; i += 2) {
+                            uint64_t v2;
+                            asm("mov.b64 %0, {%1, %2};" : "=l"(v2) : "r"(o[i]), "r"(o[i + 1]));
+                            asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(v2) : "l"(v2), "l"(alpha2));
+                            asm("mov.b64 {%0, %1}, %2;" : "=r"(o[i]), "=r"(o[i + 1]) : "l"(v2));
+                        }
+                        ptx::tmem_st32<0>(o_addr + 32 * c, o);
+                        ptx::tmem_wait_st();   // the store reads o[] asynchronously: not before this may o[] be reused
+                    }
+                    const uint32_t lcol = ptx::tmem_ld1(o_addr + 128);
+                    ptx::tmem_wait_ld();
+                    ptx::tmem_st1(o_addr + 128, __float_as_uint(__uint_as_float(lcol) * alpha));
+                    ptx::tmem_wait_st();
+                    ptx::tc_fence_before_sync();
+                }
+            }
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&sm->o_ready[sb]);
+        }
+    }
     } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 192;");
     const int quarter = warp & 3;                       // TMEM lane quarter this warp may touch
     const int group = (warp - 4) >> 2;                  // group 0 takes the even KV tiles, group 1 the odd ones
     const uint32_t row = quarter * 32 + lane;           // row inside the query tile: one thread owns one row
@@ -409,24 +471,25 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             ptx::tc_fence_after_sync();
             float r[128];
             float bmax[4];
+            bool have_prev, have_p;
             {
-                uint32_t sr[128];
                 const uint32_t s_addr = tmem + lane_base + kColS + 128 * sb;
-                ptx::tmem_ld32<0>(s_addr, sr);
-                ptx::tmem_ld32<32>(s_addr + 32, sr);
-                ptx::tmem_ld32<64>(s_addr + 64, sr);
-                ptx::tmem_ld32<96>(s_addr + 96, sr);
+                ptx::tmem_ld32f<0>(s_addr, r);
+                ptx::tmem_ld32f<32>(s_addr + 32, r);
+                ptx::tmem_ld32f<64>(s_addr + 64, r);
+                ptx::tmem_ld32f<96>(s_addr + 96, r);
+                // polls whose answers are needed later travel while the scores do
+                have_prev = j == 0 || ptx::mbar_try_wait(&sm->x_bar[sb ^ 1][quarter], static_cast<uint32_t>(((j - 1) >> 1) & 1));
+                have_p = ptx::mbar_try_wait(&sm->p_empty[sb], ph2 ^ 1u);
                 ptx::tmem_wait_ld();
                 ptx::tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&sm->s_empty[sb]);
                 const int64_t key0 = j * kTile;
-                if (key0 + 127 > limit) {
+                if (key0 + 127 > limit) {     // diagonal or ragged tile: keys past the row's limit are masked in place
 #pragma unroll
-                    for (int i = 0; i < 128; ++i) r[i] = key0 + i > limit ? -INFINITY : __uint_as_float(sr[i]);
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 128; ++i) r[i] = __uint_as_float(sr[i]);
+                    for (int i = 0; i < 128; ++i)
+                        if (key0 + i > limit) r[i] = -INFINITY;
                 }
             }
 #pragma unroll
@@ -435,7 +498,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             // ---- running row maximum (Eq. rowmax-update): handed over from the group that owns tile j-1
             float m_prev = -INFINITY;
             if (j > 0) {
-                if (!wait_all(&sm->x_bar[sb ^ 1][quarter], static_cast<uint32_t>(((j - 1) >> 1) & 1), sm, P.status)) { ok = false; break; }
+                if (!have_prev && !wait_all(&sm->x_bar[sb ^ 1][quarter], static_cast<uint32_t>(((j - 1) >> 1) & 1), sm, P.status)) { ok = false; break; }
                 m_prev = sm->runmax[sb ^ 1][row];
             }
             const float m_new = fmaxf(fmaxf(m_prev, bmax[0]), max3(bmax[1], bmax[2], bmax[3]));
@@ -447,8 +510,13 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             const bool grew = m_new > m_prev && m_prev != -INFINITY;      // history exists and must be rescaled
             const float alpha = grew ? ex2_approx(__fmul_rn(__fsub_rn(m_s_prev, m_s), K.LOG2E)) : 1.0f;
 
+            // P~V of tile j-2 finished: the P buffer is free, and so is alpha[sb] (its reader ran before that P~V)
+            if (!have_p && !wait_all(&sm->p_empty[sb], ph2 ^ 1u, sm, P.status)) { ok = false; break; }
+            sm->alpha[sb][row] = alpha;
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&sm->a_bar[sb][quarter]);
+
             // ---- probability operand (Algorithm 1 per block): codes and scales straight into the MMA operand
-            if (!wait_all(&sm->p_empty[sb], ph2 ^ 1u, sm, P.status)) { ok = false; break; }   // P~V of tile j-2 finished
             uint32_t sfword = 0;
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
@@ -474,30 +542,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 if (P.dbg.row_max) P.dbg.row_max[drow * ntile_all + j] = m_s;
             }
 
-            // ---- historical rescaling (Eq. alpha): O rows and the denominator column in TMEM
-            if (j > 0 && __any_sync(0xffffffffu, grew)) {
-                if (!wait_all(&sm->p_empty[sb ^ 1], static_cast<uint32_t>(((j - 1) >> 1) & 1), sm, P.status)) { ok = false; break; }
-                ptx::tc_fence_after_sync();
-                const uint32_t o_addr = tmem + lane_base + kColO;
-                uint32_t o[64];
-#pragma unroll
-                for (int c = 0; c < 2; ++c) {
-                    ptx::tmem_ld32<0>(o_addr + 64 * c, o);
-                    ptx::tmem_ld32<32>(o_addr + 64 * c + 32, o);
-                    ptx::tmem_wait_ld();
-#pragma unroll
-                    for (int i = 0; i < 64; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                    ptx::tmem_st32<0>(o_addr + 64 * c, o);
-                    ptx::tmem_st32<32>(o_addr + 64 * c + 32, o);
-                    ptx::tmem_wait_st();   // the stores read o[] asynchronously: not before this may o[] be reused
-                }
-                const uint32_t lcol = ptx::tmem_ld1(o_addr + 128);
-                ptx::tmem_wait_ld();
-                ptx::tmem_st1(o_addr + 128, __float_as_uint(__uint_as_float(lcol) * alpha));
-                ptx::tmem_wait_st();
-            }
             ptx::fence_proxy_async_smem();
-            ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&sm->p_full[sb]);
         }

@@ -19,6 +19,19 @@ enum Producer : int { kEfq = 0, kEtq4 = 1, kEtq6 = 2 };
 constexpr int kSegCols = 1024;       // columns per warp task
 constexpr int kWarpsPerCta = 8;
 
+__device__ __forceinline__ float fma_sat(float a, float b, float c)
+{
+    float d;
+    asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float fma_rm(float a, float b, float c)
+{
+    float d;
+    asm("fma.rm.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
 template <int PRODUCER>
 __device__ __forceinline__ void produce_block(const float (&r)[4], float m_s, const ProducerConsts& K,
                                               uint32_t& code16, uint32_t& byte)
@@ -29,9 +42,16 @@ __device__ __forceinline__ void produce_block(const float (&r)[4], float m_s, co
         rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, 2));
         rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, 4));
         BlockScale s = efq_block_scale(rmax, m_s, K);
-        uint32_t c = efq_code(r[0], K.A, s.Bb) | (efq_code(r[1], K.A, s.Bb) << 4) |
-                     (efq_code(r[2], K.A, s.Bb) << 8) | (efq_code(r[3], K.A, s.Bb) << 12);
-        code16 = s.live ? c : 0u;
+        // Four codes Horner-style on the FMA pipe, bit-identical to floor(min(max(fma(r, A, Bb), 0), 7)):
+        //   w = fma.rn.sat(r, A/8, Bb/8) = clamp(v, 0, 8)/8;  a = fma.rm(w, 8, u) = u + floor(8w) for an integer
+        //   u in [2^23, 2^24);  u' = fma.rn(a, 16, -15*2^23) = 2^23 + 16 X.  Element 0 ends in the low nibble.
+        const float A8 = K.A * 0.125f, B8 = s.Bb * 0.125f;
+        float a = fma_rm(fma_sat(r[3], A8, B8), 8.0f, 8388608.0f);
+#pragma unroll
+        for (int i = 2; i >= 0; --i) a = fma_rm(fma_sat(r[i], A8, B8), 8.0f, __fmaf_rn(a, 16.0f, -125829120.0f));
+        uint32_t c = __float_as_uint(a) & 0xffffu;
+        c -= (c >> 3) & 0x1111u;            // floor(8w) = 8 only when v >= 8: that nibble is 7
+        code16 = c;                         // a block without a finite score has w = 0 everywhere
         byte = s.byte;
     } else {
         float p[4];

@@ -186,6 +186,24 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[N])
         : "r"(taddr)
         : "memory");
 }
+#define EFQ_F32(r, o)                                                                                           \
+    "=f"(r[o + 0]), "=f"(r[o + 1]), "=f"(r[o + 2]), "=f"(r[o + 3]), "=f"(r[o + 4]), "=f"(r[o + 5]),             \
+    "=f"(r[o + 6]), "=f"(r[o + 7]), "=f"(r[o + 8]), "=f"(r[o + 9]), "=f"(r[o + 10]), "=f"(r[o + 11]),           \
+    "=f"(r[o + 12]), "=f"(r[o + 13]), "=f"(r[o + 14]), "=f"(r[o + 15]), "=f"(r[o + 16]), "=f"(r[o + 17]),       \
+    "=f"(r[o + 18]), "=f"(r[o + 19]), "=f"(r[o + 20]), "=f"(r[o + 21]), "=f"(r[o + 22]), "=f"(r[o + 23]),       \
+    "=f"(r[o + 24]), "=f"(r[o + 25]), "=f"(r[o + 26]), "=f"(r[o + 27]), "=f"(r[o + 28]), "=f"(r[o + 29]),       \
+    "=f"(r[o + 30]), "=f"(r[o + 31])
+// the same load with float destinations (FP32 accumulator columns), so that no register copies are needed
+template <int O, int N>
+__device__ __forceinline__ void tmem_ld32f(uint32_t taddr, float (&r)[N])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : EFQ_F32(r, O)
+        : "r"(taddr)
+        : "memory");
+}
 template <int O, int N>
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[N])
 {
