@@ -36,6 +36,9 @@ UNIT = "TFLOP/s"
 NOMINAL_FP4_OVER_BF16 = 4.0          # dense FP4 : dense bf16 tensor throughput on B200 (9 : 2.25 PFLOP/s)
 FALLBACK_BF16_TFLOPS = 1590.0
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the fused kernel, from the ncu capture summarised in
+# profiles/attention_fwd_qwen3_8b_16k.md (a single-pass capture at full size)
+NCU_DRAM_BYTES_PER_LAUNCH = {"qwen3_8b_16k": 56195840 + 216487168}
 
 
 def workload_case(name: str) -> inputs.AttentionCase:
@@ -77,7 +80,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                                          "-i", str(self.gpu), "-lms", "100"], stdout=subprocess.PIPE,
+                                          "-i", str(self.gpu), "-lms", "20"], stdout=subprocess.PIPE,
                                          stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -315,6 +318,33 @@ def run_cuda(args):
         stage = {"workload": "probgen 4096x16384 fp32 (device-generated N(0,9), timing only)", "bytes_per_launch": nbytes,
                  "efq_ms": t_efq, "efq_gbs": nbytes / t_efq / 1e6, "etq_ms": t_etq, "etq_gbs": nbytes / t_etq / 1e6}
 
+    # tensor-pipe and in-SM microbenchmarks (context for the roofline numbers)
+    micro = None
+    if rank == 0 and not args.skip_stage:
+        sms = torch.cuda.get_device_properties(dev).multi_processor_count
+        sink = torch.zeros(sms, dtype=torch.int32, device=dev)
+        iters = 8192
+        for _ in range(2):
+            binding.efq_fp4_mma_peak_probe(sink, sms, iters)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        fl = binding.efq_fp4_mma_peak_probe(sink, sms, iters)
+        b.record(stream)
+        torch.cuda.synchronize()
+        peak_ms = a.elapsed_time(b)
+        ok = bool((sink.cpu().numpy().view(np.uint32) != 0xdeadbeef).all())
+        per_clk = {}
+        for name, prod in (("efq", 0), ("etq", 1)):
+            binding.efq_stage_microbench(prod, 2 * sms, 200)
+            cyc = binding.efq_stage_microbench(prod, 2 * sms, 2000)
+            torch.cuda.synchronize()
+            per_clk[name] = 2 * 256 * 32 * 2000 / float(cyc.double().mean())
+        micro = {"fp4_mma_only_tflops": fl / (peak_ms * 1e-3) / 1e12 if ok else None, "fp4_mma_only_ms": peak_ms,
+                 "fp4_mma_shape": "128x256x64 kind::mxf4, one CTA per SM, %d MMAs" % iters,
+                 "stage_in_sm_elements_per_clk_per_sm": per_clk,
+                 "stage_in_sm_note": "register-resident scores, 16 warps/SM, includes one add per element of loop overhead"}
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -325,16 +355,12 @@ def run_cuda(args):
     value = whole_job_tflops(flops, ms_step, world)
     main_tflops = flops / (ms_main * 1e-3) / 1e12
     fp4_peak = peaks["bf16_sustained"] * NOMINAL_FP4_OVER_BF16
-    traffic = None
-    tpath = os.path.join(ROOT, "profiles", "attention_fwd_traffic.json")
-    if os.path.exists(tpath):
-        with open(tpath) as f:
-            traffic = json.load(f).get(args.workload)
+    traffic = NCU_DRAM_BYTES_PER_LAUNCH.get(args.workload)
 
     cpu_baseline = None
     if world == 1 and not args.skip_cpu_baseline:
         q32, k32, v32 = (inputs.bf16_bits_to_f32(t) for t in (qb, kb, vb))
-        n_rows = 4 * args.oracle_rows
+        n_rows = 32 * args.oracle_rows
         cv, csec, cores = time_oracle(case, q32, k32, v32, n_rows, 3, 1)
         cpu_baseline = {"value": cv, "unit": UNIT, "cores": cores, "kind": "oracle",
                         "sample": f"3 steps of {n_rows} seeded query rows (all heads), EFQ path, {csec:.2f} s per step"}
@@ -359,6 +385,7 @@ def run_cuda(args):
         "exp_then_quantize": {"value": flops / (etq_ms_step * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": etq_ms_step,
                               "main_kernel_ms": etq_ms_main, "efq_speedup": etq_ms_step / ms_step},
         "stage": stage,
+        "microbench": micro,
     }
     print(json.dumps(line))
     if world > 1:
@@ -373,7 +400,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="qwen3_8b_16k")
     ap.add_argument("--oracle-rows", type=int, default=2048,
-                    help="query rows the oracle computes per step (reference arm); the cpu_baseline leg uses 4x")
+                    help="query rows the oracle computes per step (reference arm); the cpu_baseline leg uses 32x")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-stage", action="store_true")
     args = ap.parse_args()

@@ -182,12 +182,21 @@ efq_status_t efq_attention_fwd_static(const void* q, const void* k, const void* 
  * EFQ_ERR_CUDA if the stream reports an error. */
 efq_status_t efq_poll_status(void* workspace, void* stream);
 
-/* Dense FP4 tensor-pipe microbenchmark: `iters` back-to-back 128x256x64 block-scaled E2M1 MMAs
- * per CTA on operands resident in shared memory, one CTA per SM.  Writes nothing but a
- * checksum word per CTA to `sink` (u32 [num_ctas]).  Used to measure the MMA-only FP4 rate
- * that the fused forward's tensor-pipe fraction is quoted against.  Returns the FLOPs per
- * launch through *flops. */
+/* Dense FP4 tensor-pipe microbenchmark: `iters` back-to-back 128x256x64 block-scaled E2M1 MMAs per CTA on
+ * operands resident in shared memory (launch one CTA per SM).  Writes one word per CTA to `sink`
+ * (u32 [num_ctas], device; 0xdeadbeef marks a CTA whose bounded wait expired) and the FLOPs of the launch to
+ * *flops (host).  The caller times the launch; FLOPs / time is the MMA-only FP4 rate that the fused forward's
+ * tensor-pipe fraction can be quoted against. */
 efq_status_t efq_fp4_mma_peak_probe(uint32_t* sink, int num_ctas, int iters, double* flops, void* stream);
+
+/* In-SM microbenchmark of the probability producers (Algorithm 1 versus exp-then-quantize) on register-resident
+ * scores: 256 threads per CTA, each coding one 32-key block per iteration, no memory traffic.
+ *   producer 0 = EFQ (params or EFQ-Mean), 1 = exp-then-quantize scale4, 2 = scale6
+ *   sink    u32 [num_ctas * 256], device (keeps the work alive)
+ *   cycles  i64 [num_ctas], device: clock cycles CTA c spent on its `iters` iterations
+ * Elements per clock per SM = resident CTAs per SM * 256 * 32 * iters / cycles. */
+efq_status_t efq_stage_microbench(int producer, const efq_params_t* params, int num_ctas, int iters, uint32_t* sink,
+                                  long long* cycles, void* stream);
 
 const char* efq_status_string(efq_status_t status);
 

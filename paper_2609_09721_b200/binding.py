@@ -24,7 +24,7 @@ STATIC_SCRATCH_BYTES = 4 << 20
 EXPORTS = ["efq_probgen", "exp_then_quantize_probgen", "efq_attention_workspace_bytes", "efq_attention_fwd",
            "exp_then_quantize_attention_fwd", "efq_quantize_qkv", "efq_attention_fwd_quantized",
            "efq_attention_fwd_host", "efq_attention_fwd_static", "efq_poll_status",
-           "efq_fp4_mma_peak_probe", "efq_status_string", "efq_version"]
+           "efq_fp4_mma_peak_probe", "efq_stage_microbench", "efq_status_string", "efq_version"]
 
 
 class EfqParams(C.Structure):
@@ -82,6 +82,8 @@ def lib() -> C.CDLL:
         L.efq_poll_status.argtypes = [vp, vp]
         L.efq_fp4_mma_peak_probe.restype = i32
         L.efq_fp4_mma_peak_probe.argtypes = [vp, i32, i32, C.POINTER(C.c_double), vp]
+        L.efq_stage_microbench.restype = i32
+        L.efq_stage_microbench.argtypes = [i32, C.POINTER(EfqParams), i32, i32, vp, vp, vp]
         L.efq_status_string.restype = C.c_char_p
         L.efq_status_string.argtypes = [i32]
         L.efq_version.restype = C.c_char_p
@@ -289,3 +291,14 @@ def efq_fp4_mma_peak_probe(sink: torch.Tensor, num_ctas: int, iters: int, stream
     st = lib().efq_fp4_mma_peak_probe(sink.data_ptr(), int(num_ctas), int(iters), C.byref(flops), _stream(stream))
     _check(st, "efq_fp4_mma_peak_probe")
     return float(flops.value)
+
+
+def efq_stage_microbench(producer: int, num_ctas: int, iters: int, params=None, stream=None):
+    """In-SM producer microbenchmark; returns the per-CTA cycle counts (int64 CUDA tensor [num_ctas])."""
+    sink = torch.empty(num_ctas * 256, dtype=torch.int32, device="cuda")
+    cycles = torch.zeros(num_ctas, dtype=torch.int64, device="cuda")
+    p = _params(params)
+    st = lib().efq_stage_microbench(int(producer), C.byref(p) if p is not None else None, int(num_ctas), int(iters),
+                                    sink.data_ptr(), cycles.data_ptr(), _stream(stream))
+    _check(st, "efq_stage_microbench")
+    return cycles

@@ -19,5 +19,3 @@ extern "C" const char* efq_status_string(efq_status_t status)
 
 extern "C" const char* efq_version(void) { return "efq-b200 sm_100a"; }
 
-// placeholder until the microbenchmark moves into the library
-extern "C" efq_status_t efq_fp4_mma_peak_probe(uint32_t*, int, int, double*, void*) { return EFQ_ERR_UNSUPPORTED; }

@@ -90,3 +90,19 @@ def test_probgen_reports_bad_arguments():
     with pytest.raises(binding.EfqError) as e:
         binding.efq_probgen(s, rm, 1.0, (-3.06, 2.3, 1))    # LUT variant not in this entry point yet
     assert e.value.status == 2
+
+
+def test_microbenchmarks_run_and_report_sane_rates():
+    """The MMA-only FP4 loop and the in-SM producer loop finish (no expired wait) and land in a sane range."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    sink = torch.zeros(sms, dtype=torch.int32, device="cuda")
+    flops = binding.efq_fp4_mma_peak_probe(sink, sms, 256)
+    torch.cuda.synchronize()
+    assert flops == 2.0 * 128 * 256 * 64 * 256 * sms
+    assert (sink.cpu().numpy().view(np.uint32) != 0xDEADBEEF).all()
+    rates = {}
+    for prod in (0, 1):
+        cyc = binding.efq_stage_microbench(prod, 2 * sms, 500)
+        torch.cuda.synchronize()
+        rates[prod] = 2 * 256 * 32 * 500 / float(cyc.double().mean())
+    assert 5.0 < rates[1] < rates[0] < 64.0     # elements per clock per SM; exp-then-quantize is MUFU-bound
