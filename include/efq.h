@@ -198,6 +198,15 @@ efq_status_t efq_fp4_mma_peak_probe(uint32_t* sink, int num_ctas, int iters, dou
 efq_status_t efq_stage_microbench(int producer, const efq_params_t* params, int num_ctas, int iters, uint32_t* sink,
                                   long long* cycles, void* stream);
 
+/* Test hook for the bounded-wait path (no GPU fault is involved): efq_attention_fwd with the K/V loads left
+ * out, so that the first device-side wait on them runs out after its limit (under a second).  Every role then
+ * drains, tensor memory is released, the kernel returns normally and the status word reads
+ * EFQ_ERR_DEVICE_TIMEOUT through efq_poll_status(); `o` is undefined.  The context stays usable and the next
+ * efq_attention_fwd on the same workspace clears the status. */
+efq_status_t efq_attention_fwd_inject_timeout(const void* q, const void* k, const void* v, float* o, int B, int Hq,
+                                              int Hkv, int64_t Sq, int64_t Sk, int d, void* workspace,
+                                              size_t workspace_bytes, void* stream);
+
 const char* efq_status_string(efq_status_t status);
 
 /* Library build tag, e.g. "efq-b200 sm_100a". */

@@ -24,7 +24,8 @@ STATIC_SCRATCH_BYTES = 4 << 20
 EXPORTS = ["efq_probgen", "exp_then_quantize_probgen", "efq_attention_workspace_bytes", "efq_attention_fwd",
            "exp_then_quantize_attention_fwd", "efq_quantize_qkv", "efq_attention_fwd_quantized",
            "efq_attention_fwd_host", "efq_attention_fwd_static", "efq_poll_status",
-           "efq_fp4_mma_peak_probe", "efq_stage_microbench", "efq_status_string", "efq_version"]
+           "efq_fp4_mma_peak_probe", "efq_stage_microbench", "efq_attention_fwd_inject_timeout", "efq_status_string",
+           "efq_version"]
 
 
 class EfqParams(C.Structure):
@@ -78,6 +79,8 @@ def lib() -> C.CDLL:
         L.efq_attention_fwd_static.restype = i32
         L.efq_attention_fwd_static.argtypes = [vp, vp, vp, vp, i32, i32, i32, i64, i64, i32, i32, f32,
                                                C.POINTER(EfqParams), vp]
+        L.efq_attention_fwd_inject_timeout.restype = i32
+        L.efq_attention_fwd_inject_timeout.argtypes = [vp, vp, vp, vp, i32, i32, i32, i64, i64, i32, vp, C.c_size_t, vp]
         L.efq_poll_status.restype = i32
         L.efq_poll_status.argtypes = [vp, vp]
         L.efq_fp4_mma_peak_probe.restype = i32
@@ -302,3 +305,12 @@ def efq_stage_microbench(producer: int, num_ctas: int, iters: int, params=None, 
                                     sink.data_ptr(), cycles.data_ptr(), _stream(stream))
     _check(st, "efq_stage_microbench")
     return cycles
+
+
+def efq_attention_fwd_inject_timeout(q, k, v, o, workspace, stream=None) -> None:
+    """Test hook: the forward with K/V loads left out, so a bounded device-side wait expires (see efq.h)."""
+    B, Hq, Sq, d = q.shape
+    _, Hkv, Sk, _ = k.shape
+    st = lib().efq_attention_fwd_inject_timeout(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, Hq, Hkv, Sq,
+                                                Sk, d, workspace.data_ptr(), workspace.numel(), _stream(stream))
+    _check(st, "efq_attention_fwd_inject_timeout")

@@ -105,6 +105,7 @@ struct FwdParams {
     uint32_t* status;
     efq_debug_t dbg;
     int has_dbg;
+    int inject_skip_loads;    // test hook: the TMA thread loads Q only, so the first wait on K/V runs out
 };
 
 // Bounded wait of one thread.  Returns false on timeout (recorded in the status word) or CTA-wide abort.
@@ -218,7 +219,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const int64_t kv_tiles = P.Sk_pad / kTile;
         int s = 0;
         uint32_t ph = 0;
-        for (int64_t j = 0; j < n_tiles; ++j) {
+        for (int64_t j = 0; j < (P.inject_skip_loads ? 0 : n_tiles); ++j) {
             // Stage barriers of their own: a waiter on a barrier that other roles may complete twice before it
             // looks (S runs ahead) could not tell which completion it sees by parity.
             if (!wait1(&sm->k_empty[s], ph ^ 1u, sm, P.status)) break;
@@ -581,7 +582,7 @@ cudaError_t launch_main(bool debug, bool fix8, dim3 grid, size_t smem, cudaStrea
 efq_status_t attention_impl(const void* q, const void* k, const void* v, float* o, int B, int Hq, int Hkv, int64_t Sq,
                             int64_t Sk, int d, int causal, float softmax_scale, int producer, float tau, float h,
                             void* workspace, size_t workspace_bytes, const efq_debug_t* debug, cudaStream_t stream,
-                            bool do_quantize, bool do_forward)
+                            bool do_quantize, bool do_forward, bool inject_skip_loads = false)
 {
     if (!q || !k || !v || !o) return EFQ_ERR_INVALID_ARG;
     if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0 || Hq % Hkv != 0) return EFQ_ERR_INVALID_ARG;
@@ -622,6 +623,7 @@ efq_status_t attention_impl(const void* q, const void* k, const void* v, float* 
     P.sf_q = ws + w.qsf; P.sf_k = ws + w.ksf; P.sf_v = ws + w.vsf;
     P.o = o;
     P.status = reinterpret_cast<uint32_t*>(ws + w.status);
+    P.inject_skip_loads = inject_skip_loads ? 1 : 0;
     P.has_dbg = debug ? 1 : 0;
     if (debug) P.dbg = *debug; else P.dbg = efq_debug_t{};
 
@@ -691,6 +693,14 @@ extern "C" efq_status_t exp_then_quantize_attention_fwd(const void* q, const voi
     if (scale_mode != 0 && scale_mode != 1) return EFQ_ERR_INVALID_ARG;
     return efq::attention_impl(q, k, v, o, B, Hq, Hkv, Sq, Sk, d, causal, softmax_scale, 1 + scale_mode, 0.0f, 1.0f,
                                workspace, workspace_bytes, debug, static_cast<cudaStream_t>(stream), true, true);
+}
+
+extern "C" efq_status_t efq_attention_fwd_inject_timeout(const void* q, const void* k, const void* v, float* o, int B,
+                                                         int Hq, int Hkv, int64_t Sq, int64_t Sk, int d, void* workspace,
+                                                         size_t workspace_bytes, void* stream)
+{
+    return efq::attention_impl(q, k, v, o, B, Hq, Hkv, Sq, Sk, d, 0, 0.0f, 0, -3.06f, 2.30f, workspace, workspace_bytes,
+                               nullptr, static_cast<cudaStream_t>(stream), true, true, true);
 }
 
 extern "C" efq_status_t efq_quantize_qkv(const void* q, const void* k, const void* v, int B, int Hq, int Hkv, int64_t Sq,

@@ -189,3 +189,20 @@ def test_attention_argument_errors():
     ws = torch.empty(binding.efq_attention_workspace_bytes(1, 2, 2, 128, 128, 128), dtype=torch.uint8, device="cuda")
     binding.efq_attention_fwd(q2, k, k, workspace=ws)
     assert binding.efq_poll_status(ws) == 0
+
+
+def test_bounded_wait_expires_and_context_stays_usable(oracle):
+    """A wait that nothing satisfies (K/V never loaded) runs out after its limit: the kernel returns, the status
+    word says EFQ_ERR_DEVICE_TIMEOUT, and the next forward on the same workspace is correct."""
+    case = inputs.AttentionCase("t", 1, 1, 1, 256, 256, 128, False, 5, "iid")
+    (q, k, v), (dq, dk, dv) = _case_tensors(case)
+    shape = (1, 1, 1, 256, 256, 128)
+    ws = torch.empty(binding.efq_attention_workspace_bytes(*shape), dtype=torch.uint8, device="cuda")
+    o = torch.empty((1, 1, 256, 128), dtype=torch.float32, device="cuda")
+    binding.efq_attention_fwd_inject_timeout(dq, dk, dv, o, ws)
+    assert binding.efq_poll_status(ws) == binding.STATUS_NAMES.index("EFQ_ERR_DEVICE_TIMEOUT")
+    o = binding.efq_attention_fwd(dq, dk, dv, False, workspace=ws)
+    assert binding.efq_poll_status(ws) == 0
+    rows = _all_rows(case, 0, 0, 256)
+    want = oracle.attention_rows(q, k, v, rows, False, case.softmax_scale, "efq")
+    assert np.abs(o.cpu().numpy()[0, 0] - want).max() <= TOL_O
