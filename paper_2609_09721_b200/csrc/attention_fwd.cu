@@ -303,7 +303,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     // One warp per TMEM lane quarter.  When a row's maximum grew in tile j, its accumulator row and its
     // denominator are multiplied by alpha_j after P~V_{j-1} has landed and before P~V_j is released; this runs
     // beside the code generation of tile j instead of inside it.
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
     const int quarter = warp & 3;
     const uint32_t row = quarter * 32 + lane;
     const uint32_t o_addr = tmem + (static_cast<uint32_t>(quarter * 32) << 16) + kColO;
@@ -347,7 +347,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         }
     }
     } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 192;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 200;");
     const int quarter = warp & 3;                       // TMEM lane quarter this warp may touch
     const int group = (warp - 4) >> 2;                  // group 0 takes the even KV tiles, group 1 the odd ones
     const uint32_t row = quarter * 32 + lane;           // row inside the query tile: one thread owns one row
