@@ -96,7 +96,6 @@ struct FwdParams {
     int B, Hq, Hkv;
     int64_t Sq, Sk, Sq_pad, Sk_pad;
     int causal;
-    int producer;             // 0 EFQ, 1 ETQ scale4, 2 ETQ scale6
     ProducerConsts K;
     const uint8_t* sf_q;      // [B*Hq*Sq_pad/128][512]
     const uint8_t* sf_k;      // [B*Hkv*Sk_pad/128][512]
@@ -618,7 +617,6 @@ efq_status_t attention_impl(const void* q, const void* k, const void* v, float* 
     FwdParams P;
     P.B = B; P.Hq = Hq; P.Hkv = Hkv; P.Sq = Sq; P.Sk = Sk; P.Sq_pad = w.Sq_pad; P.Sk_pad = w.Sk_pad;
     P.causal = causal ? 1 : 0;
-    P.producer = producer;
     P.K = make_producer_consts(softmax_scale, tau, h);
     P.sf_q = ws + w.qsf; P.sf_k = ws + w.ksf; P.sf_v = ws + w.vsf;
     P.o = o;

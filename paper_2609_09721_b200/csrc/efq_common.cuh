@@ -61,15 +61,6 @@ __device__ __forceinline__ BlockScale efq_block_scale(float rmax, float m_s, con
     return s;
 }
 
-// Per-element part (steps 5-7): affine index, clip to [0,7], floor; the result is the
-// 4-bit E2M1 pattern itself (Eq. d8-index).  -inf (masked) maps to 0.
-__device__ __forceinline__ uint32_t efq_code(float r, float A, float Bb)
-{
-    float v = __fmaf_rn(r, A, Bb);
-    v = fminf(fmaxf(v, 0.0f), 7.0f);
-    return static_cast<uint32_t>(__float2int_rd(v));
-}
-
 __device__ __forceinline__ float ex2_approx(float x)
 {
     float y;

@@ -83,10 +83,6 @@ __device__ __forceinline__ void tc_fence_after_sync()
 {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 }
-__device__ __forceinline__ void named_bar_sync(uint32_t id, uint32_t threads)
-{
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
-}
 
 // ---------------------------------------------------------------- TMA
 // 2-D tiled load; x is the innermost coordinate (x * element size must be a multiple of 16 bytes).

@@ -206,3 +206,60 @@ def test_bounded_wait_expires_and_context_stays_usable(oracle):
     rows = _all_rows(case, 0, 0, 256)
     want = oracle.attention_rows(q, k, v, rows, False, case.softmax_scale, "efq")
     assert np.abs(o.cpu().numpy()[0, 0] - want).max() <= TOL_O
+
+
+def test_batch_two_and_quantized_workspace_reuse(oracle):
+    """B = 2 with GQA; the two-call form (quantise once, forward twice with different producers and parameters)
+    gives the same results as the one-call forms."""
+    case = inputs.AttentionCase("b2", 2, 4, 2, 384, 384, 128, True, 61, "k_outliers")
+    (q, k, v), (dq, dk, dv) = _case_tensors(case)
+    shape = (2, 4, 2, 384, 384, 128)
+    ws = torch.empty(binding.efq_attention_workspace_bytes(*shape), dtype=torch.uint8, device="cuda")
+    binding.efq_quantize_qkv(dq, dk, dv, ws)
+    o1 = torch.empty((2, 4, 384, 128), dtype=torch.float32, device="cuda")
+    o2 = torch.empty_like(o1)
+    o3 = torch.empty_like(o1)
+    binding.efq_attention_fwd_quantized(o1, shape, ws, True, 0.0, 0, None)
+    binding.efq_attention_fwd_quantized(o2, shape, ws, True, 0.0, 0, (-2.10, 2.70))
+    binding.efq_attention_fwd_quantized(o3, shape, ws, True, 0.0, 1, None)
+    torch.cuda.synchronize()
+    assert binding.efq_poll_status(ws) == 0
+    assert torch.equal(o1, binding.efq_attention_fwd(dq, dk, dv, True))
+    assert torch.equal(o2, binding.efq_attention_fwd(dq, dk, dv, True, 0.0, (-2.10, 2.70)))
+    assert torch.equal(o3, binding.exp_then_quantize_attention_fwd(dq, dk, dv, True))
+    rows = np.array([(b, h, i) for b in range(2) for h in range(4) for i in range(0, 384, 5)], np.int64)
+    for o, params in ((o1, MEAN), (o2, (-2.10, 2.70))):
+        want = oracle.attention_rows(q, k, v, rows, True, case.softmax_scale, "efq", *params)
+        got = o.cpu().numpy()[rows[:, 0], rows[:, 1], rows[:, 2]]
+        assert np.abs(got - want).max() <= TOL_O
+
+
+def test_explicit_softmax_scale_and_side_stream(oracle):
+    """A caller-chosen score scale and a non-default stream."""
+    case = inputs.AttentionCase("s", 1, 2, 2, 512, 512, 128, False, 62, "lowrank")
+    (q, k, v), (dq, dk, dv) = _case_tensors(case)
+    sigma = 0.05
+    st = torch.cuda.Stream()
+    st.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(st):
+        o = binding.efq_attention_fwd(dq, dk, dv, False, sigma, stream=st)
+    st.synchronize()
+    rows = np.array([(0, h, i) for h in range(2) for i in range(0, 512, 3)], np.int64)
+    want = oracle.attention_rows(q, k, v, rows, False, float(np.float32(sigma)), "efq")
+    got = o.cpu().numpy()[rows[:, 0], rows[:, 1], rows[:, 2]]
+    assert np.abs(got - want).max() <= TOL_O
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    case = inputs.AttentionCase("h", 1, 4, 1, 640, 640, 128, True, 63, "iid")
+    qb, kb, vb = inputs.make_qkv(case)
+    pin = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).pin_memory()
+    hq, hk, hv = pin(qb), pin(kb), pin(vb)
+    dq, dk, dv = torch.empty_like(hq, device="cuda"), torch.empty_like(hk, device="cuda"), torch.empty_like(hv, device="cuda")
+    do = torch.empty((1, 4, 640, 128), dtype=torch.float32, device="cuda")
+    ho = torch.empty((1, 4, 640, 128), dtype=torch.float32).pin_memory()
+    ws = torch.empty(binding.efq_attention_workspace_bytes(1, 4, 1, 640, 640, 128), dtype=torch.uint8, device="cuda")
+    binding.efq_attention_fwd_host(hq, hk, hv, ho, dq, dk, dv, do, True, 0.0, 0, None, ws)
+    torch.cuda.synchronize()
+    want = binding.efq_attention_fwd(hq.cuda(), hk.cuda(), hv.cuda(), True)
+    assert torch.equal(ho.cuda(), want)
