@@ -319,11 +319,13 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 if (any) {
                     ptx::tc_fence_after_sync();
                     uint32_t o[32];
+                    const uint64_t alpha2 = pack2(alpha, alpha);
+                    uint32_t lcol = 0;
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         ptx::tmem_ld32<0>(o_addr + 32 * c, o);
+                        if (c == 0) lcol = ptx::tmem_ld1(o_addr + 128);     // the denominator travels with the first chunk
                         ptx::tmem_wait_ld();
-                        const uint64_t alpha2 = pack2(alpha, alpha);
 #pragma unroll
                         for (int i = 0; i < 32; i += 2) {
                             uint64_t v2;
@@ -332,12 +334,9 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                             asm("mov.b64 {%0, %1}, %2;" : "=r"(o[i]), "=r"(o[i + 1]) : "l"(v2));
                         }
                         ptx::tmem_st32<0>(o_addr + 32 * c, o);
+                        if (c == 0) ptx::tmem_st1(o_addr + 128, __float_as_uint(__uint_as_float(lcol) * alpha));
                         ptx::tmem_wait_st();   // the store reads o[] asynchronously: not before this may o[] be reused
                     }
-                    const uint32_t lcol = ptx::tmem_ld1(o_addr + 128);
-                    ptx::tmem_wait_ld();
-                    ptx::tmem_st1(o_addr + 128, __float_as_uint(__uint_as_float(lcol) * alpha));
-                    ptx::tmem_wait_st();
                     ptx::tc_fence_before_sync();
                 }
             }
