@@ -53,11 +53,16 @@ __device__ __forceinline__ BlockScale efq_block_scale(float rmax, float m_s, con
 {
     BlockScale s;
     s.live = rmax != -INFINITY;
-    float Mb = __fsub_rn(__fmul_rn(K.sigma, rmax), m_s);
-    float kf = floorf(__fmaf_rn(Mb, K.LOG2E, K.L2_29));
-    kf = fminf(fmaxf(kf, -127.0f), 127.0f);
+    const float Mb = __fsub_rn(__fmul_rn(K.sigma, rmax), m_s);
+    // k = clamp(floor(t), -127, 127) = floor(clamp(t, -127, 127)); the floor by a round-down add of 1.5 * 2^23
+    // (exact for |t| < 2^22), which also leaves k in the low mantissa bits: no conversion instruction needed.
+    float t = __fmaf_rn(Mb, K.LOG2E, K.L2_29);
+    t = fminf(fmaxf(t, -127.0f), 127.0f);          // a NaN (block and row both without a finite score) becomes -127
+    float km;
+    asm("add.rm.f32 %0, %1, %2;" : "=f"(km) : "f"(t), "f"(12582912.0f));
+    const float kf = __fsub_rn(km, 12582912.0f);
     s.Bb = __fmaf_rn(-K.h, m_s, __fmaf_rn(-K.HL2, kf, K.C1));
-    s.byte = s.live ? static_cast<uint32_t>(static_cast<int>(kf) + 127) : 0u;
+    s.byte = s.live ? (__float_as_uint(km) - 0x4B400000u + 127u) : 0u;
     return s;
 }
 
