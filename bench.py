@@ -66,18 +66,41 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clock and throttle reasons while the timed region runs.
+
+    Reads NVML in-process (a query takes well under a millisecond, so even a timed region of a few tens of
+    milliseconds is covered); falls back to an `nvidia-smi -lms` child process when NVML cannot be loaded.
+    Read-only: no setting of the GPU is touched.
+    """
     QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
+    # NVML clocks-event-reason bits
+    REASON_BITS = {"sw_power_cap": 0x4, "hw_slowdown": 0x8, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40}
 
-    def __init__(self, gpu_index: int):
+    def __init__(self, gpu_index: int, period_s: float = 0.004):
         self.gpu = gpu_index
-        self.lines = []
+        self.period = period_s
+        self.samples = []          # (time, sm_mhz, sm_max_mhz, power_w, set(reasons))
         self.proc = None
         self.thread = None
+        self.stop_flag = threading.Event()
+        self.source = None
+        self.nvml = None
+        self.handle = None
 
     def start(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(self.gpu)
+            self.nvml = pynvml
+            self.source = "nvml"
+            self.thread = threading.Thread(target=self._poll_nvml, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.nvml = None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
                                           "-i", str(self.gpu), "-lms", "20"], stdout=subprocess.PIPE,
@@ -85,43 +108,78 @@ class ClockSampler:
         except OSError:
             self.proc = None
             return
-        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.source = "nvidia-smi"
+        self.thread = threading.Thread(target=self._read_smi, daemon=True)
         self.thread.start()
 
-    def _read(self):
-        for ln in self.proc.stdout:
-            self.lines.append((time.time(), ln.strip()))
+    def _poll_nvml(self):
+        n = self.nvml
+        smax = None
+        while not self.stop_flag.is_set():
+            try:
+                if smax is None:
+                    smax = float(n.nvmlDeviceGetMaxClockInfo(self.handle, n.NVML_CLOCK_SM))
+                sm = float(n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM))
+                try:
+                    mask = int(n.nvmlDeviceGetCurrentClocksEventReasons(self.handle))
+                except Exception:
+                    mask = int(n.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
+                try:
+                    power = n.nvmlDeviceGetPowerUsage(self.handle) / 1000.0
+                except Exception:
+                    power = float("nan")
+                reasons = {name for name, bit in self.REASON_BITS.items() if mask & bit}
+                self.samples.append((time.time(), sm, smax, power, reasons))
+            except Exception:
+                pass
+            time.sleep(self.period)
 
-    def stop(self, t0: float, t1: float):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=2)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
-        sm, smax, reasons, power = [], [], set(), []
+    def _read_smi(self):
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ts, ln in self.lines:
-            if ts < t0 - 0.05 or ts > t1 + 0.05:
-                continue
+        for ln in self.proc.stdout:
+            ts = time.time()
             f = [x.strip() for x in ln.split(",")]
             if len(f) < 9:
                 continue
             try:
-                sm.append(float(f[1]))
-                smax.append(float(f[2]))
-                power.append(float(f[3]))
+                sm, smax, power = float(f[1]), float(f[2]), float(f[3])
             except ValueError:
                 continue
-            for name, val in zip(names, f[5:9]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
-        if not sm:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples inside the timed region"]}
-        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(smax), "reasons": sorted(reasons),
-                "power_w_max": max(power), "samples": len(sm)}
+            reasons = {name for name, val in zip(names, f[5:9]) if val.lower().startswith("active")}
+            self.samples.append((ts, sm, smax, power, reasons))
+
+    def stop(self, t0: float, t1: float):
+        if self.source is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no clock source (NVML and nvidia-smi unavailable)"]}
+        if self.source == "nvml":
+            self.stop_flag.set()
+            self.thread.join(timeout=2)
+            try:
+                self.nvml.nvmlShutdown()
+            except Exception:
+                pass
+        else:
+            time.sleep(0.15)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        return summarize_clock_samples(self.samples, t0, t1, self.source)
+
+
+def summarize_clock_samples(samples, t0, t1, source):
+    """Median SM clock, max clock and the union of throttle reasons over the samples taken in [t0, t1]."""
+    inside = [s for s in samples if t0 <= s[0] <= t1]
+    if not inside:
+        return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples inside the timed region"], "source": source}
+    reasons = set()
+    for s in inside:
+        reasons |= s[4]
+    power = [s[3] for s in inside if s[3] == s[3]]
+    return {"sm_mhz": statistics.median(s[1] for s in inside), "sm_max_mhz": max(s[2] for s in inside),
+            "reasons": sorted(reasons), "power_w_max": max(power) if power else None, "samples": len(inside),
+            "source": source}
 
 
 # ------------------------------------------------------------------------------------------

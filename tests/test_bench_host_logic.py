@@ -73,3 +73,18 @@ def test_reference_arm_runs_on_rank0_only():
     assert line["impl"] == "reference" and line["unit"] == "TFLOP/s" and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
     assert line["config"]["workload"] == "single_head"
+
+
+def test_clock_summary_keeps_only_samples_inside_the_timed_region():
+    import bench
+    samples = [(9.0, 500.0, 1965.0, 100.0, {"hw_slowdown"}),        # before the region: ignored
+               (10.1, 1965.0, 1965.0, 700.0, set()),
+               (10.2, 1950.0, 1965.0, 900.0, {"sw_power_cap"}),
+               (10.3, 1965.0, 1965.0, float("nan"), set()),
+               (11.5, 300.0, 1965.0, 90.0, {"sw_thermal_slowdown"})]  # after the region: ignored
+    out = bench.summarize_clock_samples(samples, 10.0, 11.0, "nvml")
+    assert out["sm_mhz"] == 1965.0 and out["sm_max_mhz"] == 1965.0
+    assert out["reasons"] == ["sw_power_cap"]
+    assert out["samples"] == 3 and out["power_w_max"] == 900.0
+    empty = bench.summarize_clock_samples(samples, 20.0, 21.0, "nvml")
+    assert empty["sm_mhz"] is None and "no samples" in empty["reasons"][0]
