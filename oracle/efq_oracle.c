@@ -167,7 +167,12 @@ typedef struct {
     float sigma;  /* score scale as given            */
     float LOG2E;  /* fl32(1 / ln 2)                  */
     float L2_29;  /* fl32(log2(2/9))                 */
+    int top;      /* largest index of the affine rule: 7 (Eq. d8-index) or 15 (16-level index of the LUT variant) */
+    int fold;     /* 1: the index goes through the 16 -> 8 folding table */
 } efq_consts;
+
+/* Folding table of the LUT variant (Sec. "EFQ-Softmax-LUT Variant"): 16-level index -> E2M1 code. */
+static const uint8_t C16[16] = {0, 1, 1, 1, 1, 1, 2, 2, 3, 3, 4, 5, 5, 6, 7, 7};
 
 static efq_consts make_consts(float sigma, float tau, float h)
 {
@@ -179,8 +184,35 @@ static efq_consts make_consts(float sigma, float tau, float h)
     k.sigma = sigma;
     k.LOG2E = (float)(1.0 / log(2.0));
     k.L2_29 = (float)(log(2.0 / 9.0) / log(2.0));
+    k.top = 7;
+    k.fold = 0;
     return k;
 }
+
+/* LUT variant: the same scale rule, the index rule with the fixed pair tau16 = ln(1/24), h16 = 14 / ln 24 and
+ * sixteen levels, then the folding table.  tau16 and h16 enter in double; the FP32 constants are rounded once. */
+static efq_consts make_consts_lut(float sigma)
+{
+    const double h16 = 14.0 / log(24.0), tau16 = log(1.0 / 24.0);
+    efq_consts k;
+    k.A = (float)((double)sigma * h16);
+    k.HL2 = (float)(h16 * log(2.0));
+    k.C1 = (float)(1.0 - h16 * (log(6.0) + tau16));
+    k.h = (float)h16;
+    k.sigma = sigma;
+    k.LOG2E = (float)(1.0 / log(2.0));
+    k.L2_29 = (float)(log(2.0 / 9.0) / log(2.0));
+    k.top = 15;
+    k.fold = 1;
+    return k;
+}
+
+/* producer ids: 0 = EFQ, 1 = exp-then-quantize scale4, 2 = exp-then-quantize scale6, 3 = EFQ-LUT */
+static efq_consts consts_for(int producer, float sigma, float tau, float h)
+{
+    return producer == 3 ? make_consts_lut(sigma) : make_consts(sigma, tau, h);
+}
+static int is_efq(int producer) { return producer == 0 || producer == 3; }
 
 /* Algorithm 1 for one block of n <= 32 raw scores r_t (before the score scale sigma),
  * with m_s = the row maximum in scaled units (fl32(sigma * max r) inside attention, the
@@ -193,6 +225,7 @@ static efq_consts make_consts(float sigma, float tau, float h)
  *   v_t  = fma(r_t, sigma h, B_b)   == (z_t - tau) h + 1 with z_t of Eq. z-def   step 5
  *   c_t  = floor(min(max(v_t, 0), 7))                                step 6 (Eq. d8-index;
  *          the +1 sits inside the floor, clip and floor commute on [0,7])
+ * LUT variant: the same sequence with (tau16, h16), j_t = floor(min(max(v_t, 0), 15)), c_t = C16[j_t].
  * A block whose maximum is -inf (fully masked) gets byte 0 and all-zero codes.
  * Returns the E8M0 byte k_b + 127 and writes n codes (0..7, one per byte). */
 static uint8_t efq_block(const float* r, int n, float m_s, const efq_consts* K, uint8_t* code)
@@ -213,8 +246,9 @@ static uint8_t efq_block(const float* r, int n, float m_s, const efq_consts* K, 
     for (int t = 0; t < n; ++t) {
         float v = fmaf(r[t], K->A, Bb);
         if (!(v > 0.0f)) v = 0.0f; /* also catches -inf */
-        if (v > 7.0f) v = 7.0f;
-        code[t] = (uint8_t)(int)floorf(v);
+        if (v > (float)K->top) v = (float)K->top;
+        int idx = (int)floorf(v);
+        code[t] = K->fold ? C16[idx] : (uint8_t)idx;
     }
     return (uint8_t)((int)kf + 127);
 }
@@ -264,21 +298,21 @@ static void pack_codes(const uint8_t* code, int n, uint8_t* packed /* 16 bytes *
 /* Standalone stage: (x, B, tau, h) -> (Q_P, s_P)  (paper Sec. 4.3, kernel interface)   */
 /* ---------------------------------------------------------------------------------- */
 
-/* producer: 0 = EFQ, 1 = exp-then-quantize scale4, 2 = exp-then-quantize scale6.
+/* producer: 0 = EFQ, 1 = exp-then-quantize scale4, 2 = exp-then-quantize scale6, 3 = EFQ-LUT (tau, h unused).
  * scores [rows, ld] fp32 raw; row_max [rows] in scaled units; codes [rows, nblk*16]
  * packed low nibble first; scales [rows, nblk]; nblk = ceil(cols/32). */
 void efq_oracle_probgen(const float* scores, int64_t ld, const float* row_max, int64_t rows, int64_t cols,
                         float sigma, float tau, float h, int producer, uint8_t* codes, uint8_t* scales)
 {
     int64_t nblk = (cols + MXB - 1) / MXB;
-    efq_consts K = make_consts(sigma, tau, h);
+    efq_consts K = consts_for(producer, sigma, tau, h);
 #pragma omp parallel for schedule(static)
     for (int64_t i = 0; i < rows; ++i) {
         uint8_t c[MXB];
         for (int64_t b = 0; b < nblk; ++b) {
             int n = cols - b * MXB < MXB ? (int)(cols - b * MXB) : MXB;
             const float* r = scores + i * ld + b * MXB;
-            uint8_t sb = producer == 0 ? efq_block(r, n, row_max[i], &K, c)
+            uint8_t sb = is_efq(producer) ? efq_block(r, n, row_max[i], &K, c)
                                        : etq_block(r, n, row_max[i], sigma, producer - 1, c);
             scales[i * nblk + b] = sb;
             pack_codes(c, n, codes + (i * nblk + b) * (MXB / 2));
@@ -323,7 +357,7 @@ static void online_row(const float* r, int64_t n_keys, const float* vhat, int d,
         l *= alpha;
         for (int64_t t = t0; t < t1; t += MXB) {
             int n = t1 - t < MXB ? (int)(t1 - t) : MXB;
-            uint8_t sb = producer == 0 ? efq_block(r + t, n, m_s, K, c)
+            uint8_t sb = is_efq(producer) ? efq_block(r + t, n, m_s, K, c)
                                        : etq_block(r + t, n, m_s, K->sigma, producer - 1, c);
             if (scales_out) scales_out[t / MXB] = sb;
             if (codes_out) pack_codes(c, n, codes_out + (t / MXB) * (MXB / 2));
@@ -351,7 +385,7 @@ void efq_oracle_online_codes(const float* scores, int64_t ld, int64_t rows, int6
 {
     int64_t nblk = (n_keys + MXB - 1) / MXB;
     int64_t ntile = (n_keys + Bc - 1) / Bc;
-    efq_consts K = make_consts(sigma, tau, h);
+    efq_consts K = consts_for(producer, sigma, tau, h);
 #pragma omp parallel for schedule(dynamic, 4)
     for (int64_t i = 0; i < rows; ++i) {
         double dummy[1];
@@ -377,7 +411,7 @@ static int64_t visible_keys(int64_t i, int64_t Sq, int64_t Sk, int causal)
 
 /* q [B,Hq,Sq,d], k, v [B,Hkv,Sk,d] as fp32 (exact widenings of the bf16 inputs).
  * rows [n_rows, 3] = (b, head, query index).  path: 0 = exact (double, unquantised),
- * 1 = EFQ, 2 = ETQ scale4, 3 = ETQ scale6.  out [n_rows, d] fp32.
+ * 1 = EFQ, 2 = ETQ scale4, 3 = ETQ scale6, 4 = EFQ-LUT.  out [n_rows, d] fp32.
  * Optional dumps (NULL to skip), each row-major over the sampled rows:
  *   raw [n_rows, Sk] (-inf where masked), codes [n_rows, nblk*16], scales [n_rows, nblk],
  *   ms [n_rows, ntile]. */
@@ -391,7 +425,7 @@ void efq_oracle_attention_rows(const float* q, const float* k, const float* v,
     int group = Hq / Hkv;
     int64_t nblk = (Sk + MXB - 1) / MXB;
     int64_t ntile = (Sk + Bc - 1) / Bc;
-    efq_consts K = make_consts(sigma, tau, h);
+    efq_consts K = consts_for(path - 1, sigma, tau, h);
 
     /* which (b, kv head) pairs are needed */
     int n_kv = B * Hkv;

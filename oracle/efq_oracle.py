@@ -3,7 +3,8 @@
 All arrays are numpy, host memory.  bf16 inputs are passed as float32 (exact widenings).
 Paths: "exact" (double softmax attention on the unquantised inputs), "efq" (Algorithm 2
 with Algorithm 1 as producer), "etq" (exp-then-quantize producer, block maximum scaled
-into [4, 8)), "etq6" (same with the block maximum scaled into (3, 6]).
+into [4, 8)), "etq6" (same with the block maximum scaled into (3, 6]), "efq_lut" (Algorithm 1 with
+the 16-level index and the folding table of the LUT variant; tau and h are not used).
 """
 from __future__ import annotations
 
@@ -15,8 +16,8 @@ from . import build as _build
 
 _lib = None
 
-PATHS = {"exact": 0, "efq": 1, "etq": 2, "etq6": 3}
-PRODUCERS = {"efq": 0, "etq": 1, "etq6": 2}
+PATHS = {"exact": 0, "efq": 1, "etq": 2, "etq6": 3, "efq_lut": 4}
+PRODUCERS = {"efq": 0, "etq": 1, "etq6": 2, "efq_lut": 3}
 
 # (tau, h) operating points printed in the paper's "Parameter selection" paragraph.
 EFQ_MEAN = (-3.06, 2.30)

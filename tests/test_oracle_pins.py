@@ -300,7 +300,7 @@ def test_exact_path_matches_library_attention(oracle, causal):
     assert np.abs(out - want).max() < 1e-6
 
 
-@pytest.mark.parametrize("path", ["efq", "etq"])
+@pytest.mark.parametrize("path", ["efq", "etq", "efq_lut"])
 @pytest.mark.parametrize("causal", [False, True])
 def test_online_recurrence_closed_form(oracle, path, causal):
     """Unrolled recurrence: O = sum_j w_j dA_j / sum_j w_j dl_j with w_j = exp(m_j - m_last),
@@ -401,7 +401,7 @@ def test_single_visible_key_returns_its_value(oracle):
             assert np.abs(out[n] - want).max() < 1e-6
 
 
-@pytest.mark.parametrize("path", ["efq", "etq"])
+@pytest.mark.parametrize("path", ["efq", "etq", "efq_lut"])
 def test_output_is_convex_combination_and_near_exact(oracle, path):
     case, q, k, v, rows = _small_case(S=384)
     out = oracle.attention_rows(q, k, v, rows, False, case.softmax_scale, path)
@@ -418,3 +418,78 @@ def test_lut_variant_fold_table():
     c = efq_math.lut16_code(z)
     assert c.min() == 0 and c.max() == 7 and np.all(np.diff(c) >= 0)
     assert efq_math.lut16_code(np.array([math.log(1 / 24) - 1e-9]))[0] == 0
+
+
+# ---------------------------------------------------------------------------------------
+# LUT variant (Sec. "EFQ-Softmax-LUT Variant"): 16-level index, folding table
+# ---------------------------------------------------------------------------------------
+
+# The folding table steps at j = 1, 6, 8, 10, 11, 13, 14, and j >= n  <=>  z >= tau16 + (n-1)/h16, so with
+# tau16 = ln(1/24), h16 = 14/ln 24 the code is the number of thresholds 0.25 * 24^((n-1)/14) that the
+# block-normalised probability 6 e^z has reached: a closed form with no floor, no table and no (tau, h).
+LUT_STEPS = (1, 6, 8, 10, 11, 13, 14)
+LUT_THRESHOLDS = np.array([0.25 * 24.0 ** ((n - 1) / 14.0) for n in LUT_STEPS])
+
+
+def test_lut_thresholds_sit_next_to_the_e2m1_rounding_boundaries():
+    rne = np.array([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0])     # midpoints between neighbouring E2M1 values
+    assert LUT_THRESHOLDS[0] == 0.25
+    assert np.all(np.abs(LUT_THRESHOLDS / rne - 1.0) < 0.11)
+    assert abs(0.25 * 24.0 ** (14 / 14.0) - 6.0) < 1e-12        # z = 0 (p~ = 6 * 2^k) is the j = 14 | 15 boundary
+
+
+def test_lut_codes_count_thresholds(oracle):
+    rng = np.random.default_rng(11)
+    x = -rng.uniform(0, 9, (600, 32)).astype(np.float32)
+    x[:, 0] = -rng.uniform(0, 3, 600).astype(np.float32)           # block maximum
+    x[:, 0] = np.maximum(x[:, 0], x.max(axis=1))
+    c, k = _probgen_blocks(oracle, x, 0.0, 1.0, producer="efq_lut")  # (tau, h) must not matter
+    c2, k2 = _probgen_blocks(oracle, x, *MEAN, producer="efq_lut")
+    assert np.array_equal(c, c2) and np.array_equal(k, k2)
+    _, k_affine = _probgen_blocks(oracle, x, *MEAN)
+    assert np.array_equal(k, k_affine)                              # the same block scale as the main method
+    xd = x.astype(np.float64)
+    p6 = 6.0 * np.exp(xd - k.astype(np.float64) * LN2 - LN6)        # 6 e^z = e^x / 2^k
+    want = (p6[..., None] >= LUT_THRESHOLDS).sum(-1)
+    edge = (np.abs(p6[..., None] / LUT_THRESHOLDS - 1.0) < 1e-4).any(-1)
+    assert edge.mean() < 0.01
+    assert np.array_equal(c[~edge], want[~edge])
+    assert np.all(np.abs(c - want) <= 1)
+    # fp64 evaluation of the printed equations (floor + table) agrees off the knife edges too
+    z = xd - k.astype(np.float64) * LN2 - LN6
+    assert np.array_equal(efq_math.lut16_code(z)[~edge], c[~edge])
+    assert c.min() >= 0 and c.max() <= 7
+
+
+def test_lut_block_maximum_code(oracle):
+    # 6 e^{z_max} lies in [4.5, 9): the block maximum gets code 7 from 0.25 * 24^(13/14) = 4.78 on, else 6
+    M = -np.linspace(0.0, 30.0, 3001)
+    x = np.full((M.size, 32), -np.inf, np.float32)
+    x[:, 7] = M.astype(np.float32)
+    c, k = _probgen_blocks(oracle, x, *MEAN, producer="efq_lut")
+    p6 = np.exp(x[:, 7].astype(np.float64)) / np.exp2(k[:, 0].astype(np.float64))
+    assert np.all(p6 >= 4.5 * (1 - 1e-5)) and np.all(p6 < 9.0 * (1 + 1e-5))
+    edge = np.abs(p6 / LUT_THRESHOLDS[-1] - 1.0) < 1e-4
+    assert np.array_equal(c[~edge, 7], np.where(p6[~edge] >= LUT_THRESHOLDS[-1], 7, 6))
+    assert set(np.unique(c[:, 7])) == {6, 7}
+
+
+def test_lut_is_monotone_and_masked_keys_are_zero(oracle):
+    x = np.linspace(-12.0, 0.0, 64, dtype=np.float32)[None, :].repeat(2, 0)
+    x[1, ::5] = -np.inf
+    c, _ = _probgen_blocks(oracle, x, *MEAN, producer="efq_lut")
+    assert np.all(np.diff(c[0, :32]) >= 0) and np.all(np.diff(c[0, 32:]) >= 0)
+    assert np.all(c[1, ::5] == 0)
+
+
+def test_lut_attention_is_closer_to_exact_than_the_affine_rule(oracle):
+    # the finer intermediate index places the thresholds next to the nearest-rounding boundaries of E2M1
+    # (Sec. "EFQ-Softmax-LUT Variant": the accuracy-oriented comparison point)
+    case, q, k, v, rows = _small_case(S=384)
+    ex = oracle.attention_rows(q, k, v, rows, False, case.softmax_scale, "exact")
+    err = {}
+    for path in ("efq", "efq_lut", "etq"):
+        out = oracle.attention_rows(q, k, v, rows, False, case.softmax_scale, path)
+        err[path] = np.linalg.norm(out - ex) / np.linalg.norm(ex)
+    assert err["efq_lut"] < err["efq"]
+    assert err["efq_lut"] < 1.5 * err["etq"]
