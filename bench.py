@@ -287,11 +287,14 @@ def run_cuda(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    LUT = (0.0, 1.0, 1)      # efq_params_t with variant 1: the EFQ-Softmax-LUT ablation (tau, h not read)
+
     def step(producer=0, ev=None):
         binding.efq_quantize_qkv(dq, dk, dv, ws)
         if ev is not None:
             ev[0].record(stream)
-        binding.efq_attention_fwd_quantized(o, shape, ws, case.causal, 0.0, producer)
+        binding.efq_attention_fwd_quantized(o, shape, ws, case.causal, 0.0, 0 if producer == 3 else producer,
+                                            LUT if producer == 3 else None)
         if ev is not None:
             ev[1].record(stream)
 
@@ -330,6 +333,7 @@ def run_cuda(args):
     if status != 0:
         raise SystemExit(f"bench.py: device status {status} after the timed region")
     etq_ms_step, etq_ms_main, _ = timed(1, max(3, args.steps // 2), 3)
+    lut_ms_step, lut_ms_main, _ = timed(3, max(3, args.steps // 4), 3)
 
     # end to end: pinned host inputs -> device -> forward -> host output, every step
     ho = torch.empty((case.B, case.Hq, case.Sq, case.d), dtype=torch.float32).pin_memory()
@@ -373,8 +377,10 @@ def run_cuda(args):
 
         t_efq = stage_time(lambda: binding.efq_probgen(sc, rm, 1.0, None, codes, scl))
         t_etq = stage_time(lambda: binding.exp_then_quantize_probgen(sc, rm, 1.0, 0, codes, scl))
+        t_lut = stage_time(lambda: binding.efq_probgen(sc, rm, 1.0, LUT, codes, scl))
         stage = {"workload": "probgen 4096x16384 fp32 (device-generated N(0,9), timing only)", "bytes_per_launch": nbytes,
-                 "efq_ms": t_efq, "efq_gbs": nbytes / t_efq / 1e6, "etq_ms": t_etq, "etq_gbs": nbytes / t_etq / 1e6}
+                 "efq_ms": t_efq, "efq_gbs": nbytes / t_efq / 1e6, "etq_ms": t_etq, "etq_gbs": nbytes / t_etq / 1e6,
+                 "efq_lut_ms": t_lut, "efq_lut_gbs": nbytes / t_lut / 1e6}
 
     # tensor-pipe and in-SM microbenchmarks (context for the roofline numbers)
     micro = None
@@ -393,7 +399,7 @@ def run_cuda(args):
         peak_ms = a.elapsed_time(b)
         ok = bool((sink.cpu().numpy().view(np.uint32) != 0xdeadbeef).all())
         per_clk = {}
-        for name, prod in (("efq", 0), ("etq", 1)):
+        for name, prod in (("efq", 0), ("etq", 1), ("efq_lut", 3)):
             binding.efq_stage_microbench(prod, 2 * sms, 200)
             cyc = binding.efq_stage_microbench(prod, 2 * sms, 2000)
             torch.cuda.synchronize()
@@ -442,6 +448,8 @@ def run_cuda(args):
         "cpu_baseline": cpu_baseline,
         "exp_then_quantize": {"value": flops / (etq_ms_step * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": etq_ms_step,
                               "main_kernel_ms": etq_ms_main, "efq_speedup": etq_ms_step / ms_step},
+        "efq_lut": {"value": flops / (lut_ms_step * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": lut_ms_step,
+                    "main_kernel_ms": lut_ms_main, "note": "variant 1: 16-level index + folding table (accuracy ablation)"},
         "stage": stage,
         "microbench": micro,
     }

@@ -51,7 +51,13 @@ typedef enum {
 typedef struct {
     float tau;
     float h;          /* > 0 */
-    int32_t variant;  /* 0 = affine rule (Eq. d8-index); 1 = 16-level LUT variant (Sec. 3.4) */
+    int32_t variant;  /* 0 = affine rule (Eq. d8-index).
+                         1 = EFQ-Softmax-LUT (Sec. "EFQ-Softmax-LUT Variant"): the same block scale, the index
+                         j = clip_[0,15](floor((z - tau16) h16) + 1) with the fixed pair tau16 = ln(1/24),
+                         h16 = 14 / ln 24, folded by C16 = [0,1,1,1,1,1,2,2,3,3,4,5,5,6,7,7]; tau and h above
+                         are not read.  Accepted by efq_probgen, every efq_attention_fwd* entry point and (as
+                         producer 0 + variant 1) by the entry points that take a producer id.  Any other value
+                         returns EFQ_ERR_UNSUPPORTED. */
     int32_t kv_tile;  /* Bc, keys per online-softmax step; 0 = default (128).  The shifted score uses the
                          running row maximum that includes the current KV block (Algorithm 2, steps 2-3),
                          so codes depend on this width.  Must be 128 in this build. */
@@ -191,7 +197,7 @@ efq_status_t efq_fp4_mma_peak_probe(uint32_t* sink, int num_ctas, int iters, dou
 
 /* In-SM microbenchmark of the probability producers (Algorithm 1 versus exp-then-quantize) on register-resident
  * scores: 256 threads per CTA, each coding one 32-key block per iteration, no memory traffic.
- *   producer 0 = EFQ (params or EFQ-Mean), 1 = exp-then-quantize scale4, 2 = scale6
+ *   producer 0 = EFQ (params or EFQ-Mean), 1 = exp-then-quantize scale4, 2 = scale6, 3 = EFQ-LUT
  *   sink    u32 [num_ctas * 256], device (keeps the work alive)
  *   cycles  i64 [num_ctas], device: clock cycles CTA c spent on its `iters` iterations
  * Elements per clock per SM = resident CTAs per SM * 256 * 32 * iters / cycles. */

@@ -39,14 +39,6 @@ cudaError_t launch_quantize_rows(const void* x, int64_t n_heads, int64_t S, int6
 cudaError_t launch_quantize_v(const void* v, int64_t n_heads, int64_t S, int64_t S_pad, uint8_t* vt_codes, uint8_t* sf,
                               cudaStream_t stream);
 
-#ifdef EFQ_TIMELINE
-__device__ long long* g_timeline = nullptr;   // [role 0..2][tile][8] clock stamps of CTA 0 (working instrumentation)
-#define TL(role, tile, slot) do { if (blockIdx.x == 0 && (threadIdx.x & 31) == 0 && g_timeline && (tile) < 256) \
-    g_timeline[((role) * 256 + (tile)) * 8 + (slot)] = clock64(); } while (0)
-#else
-#define TL(role, tile, slot) do { } while (0)
-#endif
-
 namespace {
 
 constexpr int kTile = 128;            // query rows per CTA and keys per KV tile (Bc)
@@ -570,11 +562,15 @@ template <int PRODUCER>
 cudaError_t launch_main(bool debug, bool fix8, dim3 grid, size_t smem, cudaStream_t stream, const CUtensorMap& mq,
                         const CUtensorMap& mk, const CUtensorMap& mv, const FwdParams& P)
 {
-    if (PRODUCER != 0) fix8 = false;
-    if (debug) return fix8 ? launch_one<PRODUCER, true, true>(grid, smem, stream, mq, mk, mv, P)
-                           : launch_one<PRODUCER, true, false>(grid, smem, stream, mq, mk, mv, P);
-    return fix8 ? launch_one<PRODUCER, false, true>(grid, smem, stream, mq, mk, mv, P)
-                : launch_one<PRODUCER, false, false>(grid, smem, stream, mq, mk, mv, P);
+    if constexpr (PRODUCER != 0) {     // the 8 -> 7 fix belongs to the affine rule alone
+        return debug ? launch_one<PRODUCER, true, false>(grid, smem, stream, mq, mk, mv, P)
+                     : launch_one<PRODUCER, false, false>(grid, smem, stream, mq, mk, mv, P);
+    } else {
+        if (debug) return fix8 ? launch_one<PRODUCER, true, true>(grid, smem, stream, mq, mk, mv, P)
+                               : launch_one<PRODUCER, true, false>(grid, smem, stream, mq, mk, mv, P);
+        return fix8 ? launch_one<PRODUCER, false, true>(grid, smem, stream, mq, mk, mv, P)
+                    : launch_one<PRODUCER, false, false>(grid, smem, stream, mq, mk, mv, P);
+    }
 }
 
 efq_status_t attention_impl(const void* q, const void* k, const void* v, float* o, int B, int Hq, int Hkv, int64_t Sq,
@@ -616,7 +612,7 @@ efq_status_t attention_impl(const void* q, const void* k, const void* v, float* 
     FwdParams P;
     P.B = B; P.Hq = Hq; P.Hkv = Hkv; P.Sq = Sq; P.Sk = Sk; P.Sq_pad = w.Sq_pad; P.Sk_pad = w.Sk_pad;
     P.causal = causal ? 1 : 0;
-    P.K = make_producer_consts(softmax_scale, tau, h);
+    P.K = producer == 3 ? make_producer_consts_lut(softmax_scale) : make_producer_consts(softmax_scale, tau, h);
     P.sf_q = ws + w.qsf; P.sf_k = ws + w.ksf; P.sf_v = ws + w.vsf;
     P.o = o;
     P.status = reinterpret_cast<uint32_t*>(ws + w.status);
@@ -635,6 +631,7 @@ efq_status_t attention_impl(const void* q, const void* k, const void* v, float* 
         case 0: e = launch_main<0>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
         case 1: e = launch_main<1>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
         case 2: e = launch_main<2>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
+        case 3: e = launch_main<3>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
         default: return EFQ_ERR_INVALID_ARG;
     }
     return e == cudaSuccess ? EFQ_OK : EFQ_ERR_CUDA;
@@ -643,29 +640,27 @@ efq_status_t attention_impl(const void* q, const void* k, const void* v, float* 
 }  // namespace
 }  // namespace efq
 
-#ifdef EFQ_TIMELINE
-extern "C" int efq_dev_set_timeline(long long* buf)
-{
-    return static_cast<int>(cudaMemcpyToSymbol(efq::g_timeline, &buf, sizeof(buf)));
-}
-#endif
-
 extern "C" size_t efq_attention_workspace_bytes(int B, int Hq, int Hkv, int64_t Sq, int64_t Sk, int d)
 {
     if (!efq::shape_ok(B, Hq, Hkv, Sq, Sk, d)) return 0;
     return efq::plan_workspace(B, Hq, Hkv, Sq, Sk).total;
 }
 
-static bool read_params(const efq_params_t* params, float& tau, float& h, efq_status_t& st)
+// Producer ids inside the library: 0 = EFQ (affine rule), 1 / 2 = exp-then-quantize scale4 / scale6, 3 = EFQ-LUT.
+static bool read_params(const efq_params_t* params, float& tau, float& h, bool& lut, efq_status_t& st)
 {
     tau = -3.06f;
     h = 2.30f;
+    lut = false;
     st = EFQ_OK;
     if (params) {
-        if (params->variant != 0) { st = EFQ_ERR_UNSUPPORTED; return false; }
+        if (params->variant != 0 && params->variant != 1) { st = EFQ_ERR_UNSUPPORTED; return false; }
         if (params->kv_tile != 0 && params->kv_tile != 128) { st = EFQ_ERR_UNSUPPORTED; return false; }
-        tau = params->tau;
-        h = params->h;
+        lut = params->variant == 1;
+        if (!lut) {                 // the LUT variant has its own fixed (tau16, h16): tau and h are not read
+            tau = params->tau;
+            h = params->h;
+        }
     }
     return true;
 }
@@ -676,9 +671,10 @@ extern "C" efq_status_t efq_attention_fwd(const void* q, const void* k, const vo
                                           const efq_debug_t* debug, void* stream)
 {
     float tau, h;
+    bool lut;
     efq_status_t st;
-    if (!read_params(params, tau, h, st)) return st;
-    return efq::attention_impl(q, k, v, o, B, Hq, Hkv, Sq, Sk, d, causal, softmax_scale, 0, tau, h, workspace,
+    if (!read_params(params, tau, h, lut, st)) return st;
+    return efq::attention_impl(q, k, v, o, B, Hq, Hkv, Sq, Sk, d, causal, softmax_scale, lut ? 3 : 0, tau, h, workspace,
                                workspace_bytes, debug, static_cast<cudaStream_t>(stream), true, true);
 }
 
@@ -715,8 +711,10 @@ extern "C" efq_status_t efq_attention_fwd_quantized(float* o, int B, int Hq, int
                                                     const efq_debug_t* debug, void* stream)
 {
     float tau, h;
+    bool lut;
     efq_status_t st;
-    if (!read_params(params, tau, h, st)) return st;
+    if (!read_params(params, tau, h, lut, st)) return st;
+    if (producer == 0 && lut) producer = 3;
     const void* nz = reinterpret_cast<const void*>(16);   // operands already live in the workspace
     return efq::attention_impl(nz, nz, nz, o, B, Hq, Hkv, Sq, Sk, d, causal, softmax_scale, producer, tau, h, workspace,
                                workspace_bytes, debug, static_cast<cudaStream_t>(stream), false, true);
@@ -731,8 +729,10 @@ extern "C" efq_status_t efq_attention_fwd_host(const void* q_host, const void* k
     if (!q_host || !k_host || !v_host || !o_host || !q_dev || !k_dev || !v_dev || !o_dev) return EFQ_ERR_INVALID_ARG;
     if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0) return EFQ_ERR_INVALID_ARG;
     float tau, h;
+    bool lut;
     efq_status_t st;
-    if (!read_params(params, tau, h, st)) return st;
+    if (!read_params(params, tau, h, lut, st)) return st;
+    if (producer == 0 && lut) producer = 3;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t qb = static_cast<size_t>(B) * Hq * Sq * d * 2, kb = static_cast<size_t>(B) * Hkv * Sk * d * 2;
     if (cudaMemcpyAsync(q_dev, q_host, qb, cudaMemcpyHostToDevice, s) != cudaSuccess) return EFQ_ERR_CUDA;
@@ -792,8 +792,9 @@ extern "C" efq_status_t efq_attention_fwd_static(const void* q, const void* k, c
                                                  float softmax_scale, const efq_params_t* params, void* stream)
 {
     float tau, h;
+    bool lut;
     efq_status_t st;
-    if (!read_params(params, tau, h, st)) return st;
+    if (!read_params(params, tau, h, lut, st)) return st;
     if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0) return EFQ_ERR_INVALID_ARG;
     if (d != 128) return EFQ_ERR_UNSUPPORTED;
     const size_t need = efq_attention_workspace_bytes(B, Hq, Hkv, Sq, Sk, d);
@@ -802,6 +803,6 @@ extern "C" efq_status_t efq_attention_fwd_static(const void* q, const void* k, c
     void* scratch = nullptr;
     st = static_scratch_for_current_device(&scratch);
     if (st != EFQ_OK) return st;
-    return efq::attention_impl(q, k, v, o, B, Hq, Hkv, Sq, Sk, d, causal, softmax_scale, 0, tau, h, scratch,
+    return efq::attention_impl(q, k, v, o, B, Hq, Hkv, Sq, Sk, d, causal, softmax_scale, lut ? 3 : 0, tau, h, scratch,
                                EFQ_STATIC_SCRATCH_BYTES, nullptr, static_cast<cudaStream_t>(stream), true, true);
 }

@@ -38,6 +38,26 @@ inline ProducerConsts make_producer_consts(float sigma, float tau, float h)
     return c;
 }
 
+// LUT variant (Sec. "EFQ-Softmax-LUT Variant"): the same scale rule and the same affine form with the fixed pair
+// tau16 = ln(1/24), h16 = 14 / ln 24 (taken in double, the FP32 constants rounded once); the 16-level index then
+// goes through the folding table C16 = [0,1,1,1,1,1,2,2,3,3,4,5,5,6,7,7], held as one nibble per entry.
+constexpr uint64_t kLutFold16 = 0x7765543322111110ull;
+
+inline ProducerConsts make_producer_consts_lut(float sigma)
+{
+    ProducerConsts c;
+    const double ln2 = 0.693147180559945309417232121458, ln6 = 1.79175946922805500081247735838;
+    const double h16 = 14.0 / log(24.0), tau16 = log(1.0 / 24.0);
+    c.A = static_cast<float>(static_cast<double>(sigma) * h16);
+    c.HL2 = static_cast<float>(h16 * ln2);
+    c.C1 = static_cast<float>(1.0 - h16 * (ln6 + tau16));
+    c.h = static_cast<float>(h16);
+    c.sigma = sigma;
+    c.LOG2E = static_cast<float>(1.0 / ln2);
+    c.L2_29 = static_cast<float>(log(2.0 / 9.0) / ln2);
+    return c;
+}
+
 #ifdef __CUDACC__
 
 // Per-block part of Algorithm 1 (steps 1-3): from the block's largest raw score and the
@@ -71,6 +91,18 @@ __device__ __forceinline__ float ex2_approx(float x)
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+
+// LUT variant, one element: 16-level index j = floor(min(max(v, 0), 15)) of v = fma(r, A, Bb), folded to a code.
+//   w = fma.rn.sat(r, A/16, Bb/16) = clamp(v, 0, 16) / 16   (scaling by 2^-4 commutes with rounding)
+//   fma.rm(w, 16, 2^23) = 2^23 + floor(16 w): the index sits in the low mantissa bits, 16 only when v >= 16
+__device__ __forceinline__ uint32_t lut_code(float r, float A16, float B16)
+{
+    float w, t;
+    asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(w) : "f"(r), "f"(A16), "f"(B16));
+    asm("fma.rm.f32 %0, %1, %2, %3;" : "=f"(t) : "f"(w), "f"(16.0f), "f"(8388608.0f));
+    const uint32_t j = min(__float_as_uint(t) & 31u, 15u);
+    return static_cast<uint32_t>(kLutFold16 >> (4u * j)) & 15u;
 }
 
 // Two floats -> one byte of E2M1 (round-to-nearest-even, saturating); `lo` lands in bits 0-3.

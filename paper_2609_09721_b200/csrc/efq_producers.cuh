@@ -37,6 +37,8 @@ __device__ __forceinline__ float block_max32(const float* r)
 }
 
 // 32 scores of one microscaling block -> 16 bytes of codes + scale byte.
+// PRODUCER: 0 = EFQ (affine rule), 1 / 2 = exp-then-quantize with the block maximum in [4, 8) / (3, 6],
+// 3 = EFQ-LUT.
 //
 // EFQ (Algorithm 1), three FMA-pipe instructions per element, bit-identical to
 // c = floor(min(max(fma(r, A, Bb), 0), 7)):
@@ -72,6 +74,19 @@ __device__ __forceinline__ void produce32(const float* r, float rmax, float m_s,
             uint32_t word = __byte_perm(lo, hi, 0x5410);
             if (FIX8) word -= (word >> 3) & 0x11111111u;
             w[q] = word;   // a block without a finite score has w = 0 everywhere (sat(-inf) and sat(NaN) are 0)
+        }
+    } else if (PRODUCER == 3) {
+        // LUT variant: the same block scale, 16-level index, folding table (one element at a time: the
+        // accuracy-oriented comparison point of the paper, not the fast path)
+        BlockScale s = efq_block_scale(rmax, m_s, K);
+        byte = s.byte;
+        const float A16 = K.A * 0.0625f, B16 = s.Bb * 0.0625f;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            uint32_t word = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) word |= lut_code(r[q * 8 + i], A16, B16) << (4 * i);
+            w[q] = word;
         }
     } else {
         float p[32];

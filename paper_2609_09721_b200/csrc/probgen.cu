@@ -15,7 +15,7 @@
 
 namespace efq {
 
-enum Producer : int { kEfq = 0, kEtq4 = 1, kEtq6 = 2 };
+enum Producer : int { kEfq = 0, kEtq4 = 1, kEtq6 = 2, kEfqLut = 3 };
 
 constexpr int kSegCols = 1024;       // columns per warp task
 constexpr int kWarpsPerCta = 8;
@@ -64,6 +64,18 @@ __device__ __forceinline__ void produce_block(const float (&r)[8], float m_s, co
         uint32_t c = __byte_perm(__float_as_uint(lo), __float_as_uint(hi), 0x5410);
         c -= (c >> 3) & 0x11111111u;        // floor(8w) = 8 only when v >= 8: that nibble is 7
         code32 = c;                         // a block without a finite score has w = 0 everywhere
+        byte = s.byte;
+    } else if (PRODUCER == kEfqLut) {
+        float rmax = fmaxf(max3(r[0], r[1], r[2]), max3(r[3], r[4], r[5]));
+        rmax = max3(rmax, r[6], r[7]);
+        rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, 1));
+        rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, 2));
+        BlockScale s = efq_block_scale(rmax, m_s, K);
+        const float A16 = K.A * 0.0625f, B16 = s.Bb * 0.0625f;
+        uint32_t c = 0;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) c |= lut_code(r[u], A16, B16) << (4 * u);
+        code32 = c;
         byte = s.byte;
     } else {
         float p[8];
@@ -185,7 +197,7 @@ efq_status_t launch_probgen(int producer, const float* scores, int64_t ld, const
     if (major != 10) return EFQ_ERR_ARCH;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return EFQ_ERR_CUDA;
 
-    ProducerConsts K = make_producer_consts(sigma, tau, h);
+    ProducerConsts K = producer == kEfqLut ? make_producer_consts_lut(sigma) : make_producer_consts(sigma, tau, h);
     const int64_t n_tasks = rows * ((cols + kSegCols - 1) / kSegCols);
     int64_t ctas = (n_tasks + kWarpsPerCta - 1) / kWarpsPerCta;
     const int64_t cap = static_cast<int64_t>(sms) * 8 * 64;   // whole waves of 8 resident CTAs per SM
@@ -196,6 +208,7 @@ efq_status_t launch_probgen(int producer, const float* scores, int64_t ld, const
         case kEfq:  probgen_kernel<kEfq><<<grid, block, 0, stream>>>(scores, ld, row_max, rows, cols, K, codes, scales, a32); break;
         case kEtq4: probgen_kernel<kEtq4><<<grid, block, 0, stream>>>(scores, ld, row_max, rows, cols, K, codes, scales, a32); break;
         case kEtq6: probgen_kernel<kEtq6><<<grid, block, 0, stream>>>(scores, ld, row_max, rows, cols, K, codes, scales, a32); break;
+        case kEfqLut: probgen_kernel<kEfqLut><<<grid, block, 0, stream>>>(scores, ld, row_max, rows, cols, K, codes, scales, a32); break;
         default: return EFQ_ERR_INVALID_ARG;
     }
     return cudaGetLastError() == cudaSuccess ? EFQ_OK : EFQ_ERR_CUDA;
@@ -208,12 +221,14 @@ extern "C" efq_status_t efq_probgen(const float* scores, int64_t ld, const float
                                     uint8_t* codes, uint8_t* scales, void* stream)
 {
     float tau = -3.06f, h = 2.30f;
+    int producer = efq::kEfq;
     if (params) {
-        if (params->variant != 0) return EFQ_ERR_UNSUPPORTED;
-        tau = params->tau;
-        h = params->h;
+        if (params->variant != 0 && params->variant != 1) return EFQ_ERR_UNSUPPORTED;
+        if (params->variant == 1) producer = efq::kEfqLut;   // fixed (tau16, h16): tau and h are not read
+        tau = params->variant == 1 ? 0.0f : params->tau;
+        h = params->variant == 1 ? 1.0f : params->h;
     }
-    return efq::launch_probgen(efq::kEfq, scores, ld, row_max, rows, cols, score_scale, tau, h, codes, scales,
+    return efq::launch_probgen(producer, scores, ld, row_max, rows, cols, score_scale, tau, h, codes, scales,
                                static_cast<cudaStream_t>(stream));
 }
 

@@ -50,7 +50,7 @@ def _check_dump(oracle, case, dump, rows, params, producer="efq", want=None):
     for n, (_, _, i) in enumerate(rows):
         nt = (_visible(case, int(i)) + 127) // 128
         assert np.array_equal(ms[n, :nt], oms[n, :nt])
-    if producer == "efq":
+    if producer in ("efq", "efq_lut"):
         assert np.array_equal(scales, osc)
         assert np.array_equal(codes, oc)
     else:
@@ -124,6 +124,31 @@ def test_cross_shapes_sq_ne_sk(oracle, Sq, Sk, causal):
         assert np.all(got.reshape(2, Sq, 128)[:, : Sq - Sk] == 0.0)
 
 
+@pytest.mark.parametrize("S,Hq,Hkv,causal", [(1024, 1, 1, False), (384, 4, 2, True), (1000, 2, 1, True), (24, 1, 1, False)])
+def test_lut_variant_fused_forward(oracle, S, Hq, Hkv, causal):
+    """variant 1 (EFQ-Softmax-LUT) through the fused forward: operand bit-exact, O within tolerance."""
+    case = inputs.AttentionCase("lut", 1, Hq, Hkv, S, S, 128, causal, 90 + S, "iid")
+    (q, k, v), (dq, dk, dv) = _case_tensors(case)
+    head = Hq - 1
+    dump = binding.DebugDump(0, head, 0, S, S)
+    o = binding.efq_attention_fwd(dq, dk, dv, causal, 0.0, (0.0, 1.0, 1), debug=dump)
+    torch.cuda.synchronize()
+    rows = np.array([(0, h, i) for h in range(Hq) for i in range(S)], np.int64)
+    want_o = oracle.attention_rows(q, k, v, rows, causal, case.softmax_scale, "efq_lut")
+    got = o.cpu().numpy().reshape(-1, 128)
+    assert np.abs(got - want_o).max() <= TOL_O
+    _check_dump(oracle, case, dump, _all_rows(case, head, 0, S), MEAN, producer="efq_lut")
+    # without the dump (the production instantiation) the output is the same
+    o2 = binding.efq_attention_fwd(dq, dk, dv, causal, 0.0, (0.0, 1.0, 1))
+    torch.cuda.synchronize()
+    assert torch.equal(o, o2)
+    # and it is not the affine rule's output
+    o3 = binding.efq_attention_fwd(dq, dk, dv, causal, 0.0, None)
+    torch.cuda.synchronize()
+    if S >= 384:
+        assert not torch.equal(o, o3)
+
+
 @pytest.mark.parametrize("mode,path", [(0, "etq"), (1, "etq6")])
 def test_exp_then_quantize_path(oracle, mode, path):
     case = inputs.AttentionCase("t", 1, 4, 2, 640, 640, 128, True, 9, "k_outliers")
@@ -176,6 +201,9 @@ def test_attention_argument_errors():
     with pytest.raises(binding.EfqError) as e:
         binding.efq_attention_fwd(q, k, k)                   # Hq % Hkv != 0
     assert e.value.status == 1
+    with pytest.raises(binding.EfqError) as e:
+        binding.efq_attention_fwd(k, k, k, params=(-3.06, 2.30, 5))   # no such variant
+    assert e.value.status == 2
     q64 = torch.zeros((1, 2, 128, 64), dtype=torch.bfloat16, device="cuda")
     assert binding.efq_attention_workspace_bytes(1, 2, 2, 128, 128, 64) == 0
     with pytest.raises(binding.EfqError) as e:

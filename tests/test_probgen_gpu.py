@@ -61,6 +61,40 @@ def test_efq_probgen_full_config(oracle):
     assert hist[0] > 0.3 and hist[7] > 0.01
 
 
+@pytest.mark.parametrize("rows,cols,ld", [(64, 4096, None), (37, 1024 * 3 + 32 * 5, None), (5, 32760, 32768),
+                                          (9, 88, 96), (3, 31, 32), (1, 1, 4)])
+def test_efq_lut_probgen_bit_exact(oracle, rows, cols, ld):
+    """variant 1: 16-level index + folding table; (tau, h) in the params are not read."""
+    scores, row_max = inputs.make_score_matrix(rows, cols, seed=60 + rows)
+    if cols > 64:
+        scores[0, 40:104] = -np.inf
+    want_c, want_s = oracle.probgen(scores, row_max, 1.0, producer="efq_lut")
+    got_c, got_s = _run_gpu(binding.efq_probgen, scores, row_max, 1.0, (123.0, 0.5, 1), ld=ld)
+    assert np.array_equal(got_s, want_s)
+    assert np.array_equal(got_c, want_c)
+    # same block scale as the affine rule, other codes
+    aff_c, aff_s = oracle.probgen(scores, row_max, 1.0, -3.06, 2.30)
+    assert np.array_equal(aff_s, want_s)
+    if cols >= 1024:
+        assert not np.array_equal(aff_c, want_c)
+
+
+def test_efq_lut_probgen_full_config(oracle):
+    scores, row_max = inputs.make_score_matrix(4096, 16384, seed=2)
+    want_c, want_s = oracle.probgen(scores, row_max, 1.0, producer="efq_lut")
+    got_c, got_s = _run_gpu(binding.efq_probgen, scores, row_max, 1.0, (0.0, 1.0, 1))
+    assert np.array_equal(got_s, want_s)
+    assert np.array_equal(got_c, want_c)
+
+
+def test_probgen_unknown_variant_is_refused():
+    scores = torch.zeros((4, 64), dtype=torch.float32, device="cuda")
+    rm = torch.zeros(4, dtype=torch.float32, device="cuda")
+    with pytest.raises(binding.EfqError) as e:
+        binding.efq_probgen(scores, rm, 1.0, (-3.06, 2.30, 2))
+    assert e.value.status == 2
+
+
 @pytest.mark.parametrize("mode,name", [(0, "etq"), (1, "etq6")])
 def test_etq_probgen_statistical_parity(oracle, mode, name):
     scores, row_max = inputs.make_score_matrix(256, 4096 + 96, seed=7)
@@ -88,7 +122,7 @@ def test_probgen_reports_bad_arguments():
         binding.efq_probgen(s[:, 1:33], rm, 1.0, None)      # base pointer off by 4 bytes
     assert e.value.status == 3
     with pytest.raises(binding.EfqError) as e:
-        binding.efq_probgen(s, rm, 1.0, (-3.06, 2.3, 1))    # LUT variant not in this entry point yet
+        binding.efq_probgen(s, rm, 1.0, (-3.06, 2.3, 7))    # no such variant
     assert e.value.status == 2
 
 
