@@ -183,6 +183,36 @@ efq_status_t efq_attention_fwd_static(const void* q, const void* k, const void* 
                                       int64_t Sq, int64_t Sk, int d, int causal, float softmax_scale,
                                       const efq_params_t* params, void* stream);
 
+/* Softmax attention in FP32 on the unquantised bf16 inputs (the problem statement of Sec. 3.1 with no low-bit
+ * operand anywhere): O = softmax(scale Q K^T + mask) V, online over the keys, exponentials by expf.  This is the
+ * reference output O_ref of the calibration objective and the "exact" side of the error figures; a plain
+ * CUDA-core kernel, not a fast path.  Arguments as for efq_attention_fwd (no workspace); B * Hq <= 65535. */
+efq_status_t efq_exact_attention_fwd(const void* q, const void* k, const void* v, float* o, int B, int Hq, int Hkv,
+                                     int64_t Sq, int64_t Sk, int d, int causal, float softmax_scale, void* stream);
+
+/* The calibration objective rho = ||a - ref||_F / ||ref||_F (Sec. "Parameter Calibration"), as its two sums:
+ * on return of the stream work, sums[0] = sum (a - ref)^2 and sums[1] = sum ref^2 over n elements, both
+ * accumulated in double.  a, ref fp32 device; sums double[2] device (overwritten).  Asynchronous. */
+efq_status_t efq_relative_error(const float* a, const float* ref, int64_t n, double* sums, void* stream);
+
+/* Offline selection of (tau, h) by grid search (Algorithm 3): the operands are quantised once, then for every
+ * tau in taus (outer loop) and h in hs (inner loop) the fused EFQ forward runs on the calibration inputs and
+ * rho(tau, h) = ||O~(tau, h) - O_ref||_F / ||O_ref||_F is formed; the pair with the smallest rho wins, the first
+ * one in scan order on a tie.  The selected pair is meant to stay fixed at inference.
+ *   q, k, v, shape, causal, softmax_scale, workspace   as for efq_attention_fwd
+ *   o_ref    fp32 [B, Hq, Sq, d] device: the reference output (e.g. from efq_exact_attention_fwd)
+ *   o_tmp    fp32 [B, Hq, Sq, d] device scratch for the candidate outputs
+ *   taus, hs HOST arrays of n_tau and n_h candidates (every h > 0)
+ *   sums     double [2 * n_tau * n_h] device scratch
+ *   rho      HOST double [n_tau * n_h], row-major over (tau, h): the objective of every candidate
+ *   best_tau, best_h  HOST outputs (may be NULL)
+ * Synchronises `stream` before returning.  Errors: those of efq_attention_fwd, INVALID_ARG for empty candidate
+ * sets or null pointers, DEVICE_TIMEOUT if a bounded device-side wait expired in any forward. */
+efq_status_t efq_calibrate(const void* q, const void* k, const void* v, const float* o_ref, float* o_tmp, int B,
+                           int Hq, int Hkv, int64_t Sq, int64_t Sk, int d, int causal, float softmax_scale,
+                           const float* taus, int n_tau, const float* hs, int n_h, double* sums, double* rho,
+                           float* best_tau, float* best_h, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Synchronises `stream` and returns the device-side status word of the last forward that
  * used `workspace` (EFQ_OK, or EFQ_ERR_DEVICE_TIMEOUT if a bounded wait expired), or
  * EFQ_ERR_CUDA if the stream reports an error. */

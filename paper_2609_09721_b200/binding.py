@@ -24,6 +24,7 @@ STATIC_SCRATCH_BYTES = 4 << 20
 EXPORTS = ["efq_probgen", "exp_then_quantize_probgen", "efq_attention_workspace_bytes", "efq_attention_fwd",
            "exp_then_quantize_attention_fwd", "efq_quantize_qkv", "efq_attention_fwd_quantized",
            "efq_attention_fwd_host", "efq_attention_fwd_static", "efq_poll_status",
+           "efq_exact_attention_fwd", "efq_relative_error", "efq_calibrate",
            "efq_fp4_mma_peak_probe", "efq_stage_microbench", "efq_attention_fwd_inject_timeout", "efq_status_string",
            "efq_version"]
 
@@ -81,6 +82,14 @@ def lib() -> C.CDLL:
                                                C.POINTER(EfqParams), vp]
         L.efq_attention_fwd_inject_timeout.restype = i32
         L.efq_attention_fwd_inject_timeout.argtypes = [vp, vp, vp, vp, i32, i32, i32, i64, i64, i32, vp, C.c_size_t, vp]
+        L.efq_exact_attention_fwd.restype = i32
+        L.efq_exact_attention_fwd.argtypes = [vp, vp, vp, vp, i32, i32, i32, i64, i64, i32, i32, f32, vp]
+        L.efq_relative_error.restype = i32
+        L.efq_relative_error.argtypes = [vp, vp, i64, vp, vp]
+        L.efq_calibrate.restype = i32
+        L.efq_calibrate.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i64, i64, i32, i32, f32,
+                                    C.POINTER(C.c_float), i32, C.POINTER(C.c_float), i32, vp, C.POINTER(C.c_double),
+                                    C.POINTER(C.c_float), C.POINTER(C.c_float), vp, C.c_size_t, vp]
         L.efq_poll_status.restype = i32
         L.efq_poll_status.argtypes = [vp, vp]
         L.efq_fp4_mma_peak_probe.restype = i32
@@ -282,6 +291,51 @@ def efq_attention_fwd_static(q, k, v, causal: bool = False, softmax_scale: float
                                         C.byref(p) if p is not None else None, _stream(stream))
     _check(st, "efq_attention_fwd_static")
     return o
+
+
+def efq_exact_attention_fwd(q, k, v, causal: bool = False, softmax_scale: float = 0.0, o=None, stream=None):
+    """FP32 softmax attention on the unquantised bf16 inputs (reference output); returns o fp32 [B,Hq,Sq,d]."""
+    B, Hq, Sq, d = q.shape
+    _, Hkv, Sk, _ = k.shape
+    if o is None:
+        o = torch.empty((B, Hq, Sq, d), dtype=torch.float32, device=q.device)
+    st = lib().efq_exact_attention_fwd(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, Hq, Hkv, Sq, Sk, d,
+                                       int(bool(causal)), float(softmax_scale), _stream(stream))
+    _check(st, "efq_exact_attention_fwd")
+    return o
+
+
+def efq_relative_error(a: torch.Tensor, ref: torch.Tensor, sums: torch.Tensor = None, stream=None) -> float:
+    """rho = ||a - ref||_F / ||ref||_F of two fp32 CUDA tensors (synchronises to read the two sums)."""
+    assert a.is_cuda and ref.is_cuda and a.dtype == torch.float32 and ref.dtype == torch.float32
+    assert a.is_contiguous() and ref.is_contiguous() and a.numel() == ref.numel()
+    if sums is None:
+        sums = torch.empty(2, dtype=torch.float64, device=a.device)
+    st = lib().efq_relative_error(a.data_ptr(), ref.data_ptr(), a.numel(), sums.data_ptr(), _stream(stream))
+    _check(st, "efq_relative_error")
+    d2, r2 = (float(x) for x in sums.cpu())
+    if r2 > 0.0:
+        return (d2 / r2) ** 0.5
+    return float("inf") if d2 > 0.0 else 0.0
+
+
+def efq_calibrate(q, k, v, o_ref, taus, hs, causal: bool = False, softmax_scale: float = 0.0, workspace=None,
+                  stream=None):
+    """Grid search of (tau, h) (Algorithm 3).  Returns (rho [n_tau, n_h] as nested lists, (best_tau, best_h))."""
+    B, Hq, Hkv, Sq, Sk, d, o_tmp, workspace = _attn_args(q, k, v, None, workspace)
+    assert o_ref.is_cuda and o_ref.dtype == torch.float32 and o_ref.is_contiguous() and o_ref.shape == o_tmp.shape
+    n_tau, n_h = len(taus), len(hs)
+    ct = (C.c_float * n_tau)(*[float(t) for t in taus])
+    ch = (C.c_float * n_h)(*[float(h) for h in hs])
+    rho = (C.c_double * (n_tau * n_h))()
+    bt, bh = C.c_float(0.0), C.c_float(0.0)
+    sums = torch.empty(2 * n_tau * n_h, dtype=torch.float64, device=q.device)
+    st = lib().efq_calibrate(q.data_ptr(), k.data_ptr(), v.data_ptr(), o_ref.data_ptr(), o_tmp.data_ptr(), B, Hq, Hkv,
+                             Sq, Sk, d, int(bool(causal)), float(softmax_scale), ct, n_tau, ch, n_h, sums.data_ptr(),
+                             rho, C.byref(bt), C.byref(bh), workspace.data_ptr(), workspace.numel(), _stream(stream))
+    _check(st, "efq_calibrate")
+    table = [[rho[i * n_h + j] for j in range(n_h)] for i in range(n_tau)]
+    return table, (float(bt.value), float(bh.value))
 
 
 def efq_poll_status(workspace, stream=None) -> int:
