@@ -382,6 +382,23 @@ def run_cuda(args):
                  "efq_ms": t_efq, "efq_gbs": nbytes / t_efq / 1e6, "etq_ms": t_etq, "etq_gbs": nbytes / t_etq / 1e6,
                  "efq_lut_ms": t_lut, "efq_lut_gbs": nbytes / t_lut / 1e6}
 
+    # accuracy beside the speed: relative Frobenius error of each producer's output against FP32 attention on
+    # the unquantised inputs, on the whole benchmarked problem (reference kernel: plain CUDA cores, run once)
+    accuracy = None
+    if rank == 0 and not args.skip_error and case.flops <= 2.0e13:
+        t0 = time.time()
+        o_ref = binding.efq_exact_attention_fwd(dq, dk, dv, case.causal)
+        torch.cuda.synchronize()
+        t_ref = time.time() - t0
+        accuracy = {"metric": "||O - O_exact||_F / ||O_exact||_F, O_exact = FP32 softmax attention on the bf16 inputs",
+                    "reference_kernel_s": t_ref}
+        binding.efq_quantize_qkv(dq, dk, dv, ws)
+        for name, prod, prm in (("efq", 0, None), ("exp_then_quantize", 1, None), ("exp_then_quantize_scale6", 2, None),
+                                ("efq_lut", 0, LUT), ("efq_mmlu", 0, (-2.90, 2.00)), ("efq_balance", 0, (-2.10, 2.70))):
+            binding.efq_attention_fwd_quantized(o, shape, ws, case.causal, 0.0, prod, prm)
+            accuracy[name] = binding.efq_relative_error(o, o_ref)
+        del o_ref
+
     # tensor-pipe and in-SM microbenchmarks (context for the roofline numbers)
     micro = None
     if rank == 0 and not args.skip_stage:
@@ -450,6 +467,7 @@ def run_cuda(args):
                               "main_kernel_ms": etq_ms_main, "efq_speedup": etq_ms_step / ms_step},
         "efq_lut": {"value": flops / (lut_ms_step * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": lut_ms_step,
                     "main_kernel_ms": lut_ms_main, "note": "variant 1: 16-level index + folding table (accuracy ablation)"},
+        "accuracy": accuracy,
         "stage": stage,
         "microbench": micro,
     }
@@ -469,6 +487,7 @@ def main():
                     help="query rows the oracle computes per step (reference arm); the cpu_baseline leg uses 32x")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-stage", action="store_true")
+    ap.add_argument("--skip-error", action="store_true", help="skip the error-against-exact-attention report")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
