@@ -328,8 +328,15 @@ void efq_oracle_probgen(const float* scores, int64_t ld, const float* row_max, i
  * Walks KV tiles of width Bc in ascending order with the running maximum, producing the
  * probability operand per 32-key block and accumulating numerator and denominator from
  * that same operand.  Optional dumps: codes [nblk*16], scales [nblk], m_s per tile. */
+/* rescale_threshold T (scaled units, not in the paper; T = 0 is Algorithm 2 as printed): the maximum that shifts
+ * the scores is kept from tile to tile while the true running maximum exceeds it by at most T, and replaced by
+ * the true running maximum otherwise:
+ *     cand = max(m, tile maximum);   m <- cand  if m = -inf or T <= 0 or fl(fl(sigma cand) - fl(sigma m)) > T,
+ *                                    m unchanged otherwise.
+ * Shifted scores may then be positive (up to T); the scale rule is shift-equivariant, so only the block exponents
+ * move, and alpha = 1 for every tile that keeps m. */
 static void online_row(const float* r, int64_t n_keys, const float* vhat, int d, int64_t Bc,
-                       const efq_consts* K, int producer, double* out /* [d] */,
+                       const efq_consts* K, int producer, float rescale_threshold, double* out /* [d] */,
                        uint8_t* codes_out, uint8_t* scales_out, float* ms_out)
 {
     double* A = (double*)calloc((size_t)d, sizeof(double));
@@ -341,8 +348,17 @@ static void online_row(const float* r, int64_t n_keys, const float* vhat, int d,
     for (int64_t j = 0; j < ntile; ++j) {
         int64_t t0 = j * Bc;
         int64_t t1 = t0 + Bc < n_keys ? t0 + Bc : n_keys;
+        float cand = m_raw;
         for (int64_t t = t0; t < t1; ++t)
-            if (r[t] > m_raw) m_raw = r[t]; /* Eq. rowmax-update */
+            if (r[t] > cand) cand = r[t]; /* Eq. rowmax-update */
+        if (m_raw == -INFINITY || !(rescale_threshold > 0.0f)) {
+            m_raw = cand;
+        } else {
+            float sc = K->sigma * cand;
+            float su = K->sigma * m_raw;
+            float diff = sc - su;
+            if (diff > rescale_threshold) m_raw = cand;
+        }
         float m_s = K->sigma * m_raw;
         if (ms_out) ms_out[j] = m_s;
         if (m_raw == -INFINITY) { /* nothing visible yet: operand is all zero */
@@ -380,7 +396,7 @@ static void online_row(const float* r, int64_t n_keys, const float* vhat, int d,
  * kernel's codes bit-for-bit on the kernel's own FP32 scores).
  * scores [rows, ld]; codes [rows, nblk*16]; scales [rows, nblk]; ms [rows, ntile]. */
 void efq_oracle_online_codes(const float* scores, int64_t ld, int64_t rows, int64_t n_keys, int64_t Bc,
-                             float sigma, float tau, float h, int producer,
+                             float sigma, float tau, float h, int producer, float rescale_threshold,
                              uint8_t* codes, uint8_t* scales, float* ms)
 {
     int64_t nblk = (n_keys + MXB - 1) / MXB;
@@ -391,7 +407,7 @@ void efq_oracle_online_codes(const float* scores, int64_t ld, int64_t rows, int6
         double dummy[1];
         float zero = 0.0f;
         /* d = 0: no value accumulation */
-        online_row(scores + i * ld, n_keys, &zero, 0, Bc, &K, producer, dummy,
+        online_row(scores + i * ld, n_keys, &zero, 0, Bc, &K, producer, rescale_threshold, dummy,
                    codes + i * nblk * (MXB / 2), scales + i * nblk, ms ? ms + i * ntile : NULL);
     }
 }
@@ -417,7 +433,7 @@ static int64_t visible_keys(int64_t i, int64_t Sq, int64_t Sk, int causal)
  *   ms [n_rows, ntile]. */
 void efq_oracle_attention_rows(const float* q, const float* k, const float* v,
                                int B, int Hq, int Hkv, int64_t Sq, int64_t Sk, int d, int causal,
-                               float sigma, float tau, float h, int64_t Bc, int path,
+                               float sigma, float tau, float h, int64_t Bc, int path, float rescale_threshold,
                                const int64_t* rows, int64_t n_rows, float* out,
                                float* raw, uint8_t* codes, uint8_t* scales, float* ms)
 {
@@ -486,7 +502,7 @@ void efq_oracle_attention_rows(const float* q, const float* k, const float* v,
                 r[t] = (float)acc;
             }
             double* od = (double*)malloc(sizeof(double) * (size_t)d);
-            online_row(r, Sk, vhat, d, Bc, &K, path - 1, od,
+            online_row(r, Sk, vhat, d, Bc, &K, path - 1, rescale_threshold, od,
                        codes ? codes + n * nblk * (MXB / 2) : NULL,
                        scales ? scales + n * nblk : NULL, ms ? ms + n * ntile : NULL);
             for (int c = 0; c < d; ++c) o[c] = (float)od[c];

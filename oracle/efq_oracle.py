@@ -40,9 +40,9 @@ def lib():
         L.efq_oracle_probgen.argtypes = [fp, i64, fp, i64, i64, C.c_float, C.c_float, C.c_float,
                                          C.c_int, u8, u8]
         L.efq_oracle_online_codes.argtypes = [fp, i64, i64, i64, i64, C.c_float, C.c_float, C.c_float,
-                                              C.c_int, u8, u8, fp]
+                                              C.c_int, C.c_float, u8, u8, fp]
         L.efq_oracle_attention_rows.argtypes = [fp, fp, fp, C.c_int, C.c_int, C.c_int, i64, i64, C.c_int,
-                                                C.c_int, C.c_float, C.c_float, C.c_float, i64, C.c_int,
+                                                C.c_int, C.c_float, C.c_float, C.c_float, i64, C.c_int, C.c_float,
                                                 C.POINTER(i64), i64, fp, fp, u8, u8, fp]
         _lib = L
     return _lib
@@ -104,9 +104,10 @@ def probgen(scores: np.ndarray, row_max: np.ndarray, sigma: float = 1.0, tau: fl
 
 
 def online_codes(scores: np.ndarray, Bc: int, sigma: float, tau: float = EFQ_MEAN[0],
-                 h: float = EFQ_MEAN[1], producer: str = "efq"):
+                 h: float = EFQ_MEAN[1], producer: str = "efq", rescale_threshold: float = 0.0):
     """Online (running-maximum) code generation on given raw scores [rows, n_keys].
-    Returns (codes, scales, m_s [rows, ntile])."""
+    Returns (codes, scales, m_s [rows, ntile]).  rescale_threshold > 0 keeps the shifting maximum while the
+    true maximum exceeds it by at most that much (scaled units); 0 is Algorithm 2."""
     scores = np.ascontiguousarray(scores, dtype=np.float32)
     rows, n_keys = scores.shape
     nblk = (n_keys + 31) // 32
@@ -115,13 +116,13 @@ def online_codes(scores: np.ndarray, Bc: int, sigma: float, tau: float = EFQ_MEA
     scales = np.empty((rows, nblk), dtype=np.uint8)
     ms = np.empty((rows, ntile), dtype=np.float32)
     lib().efq_oracle_online_codes(_fp(scores), n_keys, rows, n_keys, Bc, sigma, tau, h,
-                                  PRODUCERS[producer], _u8(codes), _u8(scales), _fp(ms))
+                                  PRODUCERS[producer], rescale_threshold, _u8(codes), _u8(scales), _fp(ms))
     return codes, scales, ms
 
 
 def attention_rows(q: np.ndarray, k: np.ndarray, v: np.ndarray, rows: np.ndarray, causal: bool,
                    sigma: float, path: str = "efq", tau: float = EFQ_MEAN[0], h: float = EFQ_MEAN[1],
-                   Bc: int = 128, dumps: bool = False):
+                   Bc: int = 128, dumps: bool = False, rescale_threshold: float = 0.0):
     """Attention forward on sampled rows.  q [B,Hq,Sq,d], k/v [B,Hkv,Sk,d] float32;
     rows int64 [n, 3] of (b, head, query index).  Returns out [n, d] float32, and with
     ``dumps`` a dict of raw scores, packed codes, scale bytes and per-tile m_s."""
@@ -141,7 +142,7 @@ def attention_rows(q: np.ndarray, k: np.ndarray, v: np.ndarray, rows: np.ndarray
         scales = np.empty((n, nblk), dtype=np.uint8)
         ms = np.empty((n, (Sk + Bc - 1) // Bc), dtype=np.float32)
     lib().efq_oracle_attention_rows(_fp(q), _fp(k), _fp(v), B, Hq, Hkv, Sq, Sk, d, int(causal),
-                                    sigma, tau, h, Bc, PATHS[path],
+                                    sigma, tau, h, Bc, PATHS[path], rescale_threshold,
                                     rows.ctypes.data_as(C.POINTER(C.c_int64)), n, _fp(out),
                                     _fp(raw), _u8(codes), _u8(scales), _fp(ms))
     if dumps:

@@ -493,3 +493,82 @@ def test_lut_attention_is_closer_to_exact_than_the_affine_rule(oracle):
         err[path] = np.linalg.norm(out - ex) / np.linalg.norm(ex)
     assert err["efq_lut"] < err["efq"]
     assert err["efq_lut"] < 1.5 * err["etq"]
+
+
+# ---------------------------------------------------------------------------------------
+# thresholded rescaling (not in the paper; threshold 0 is Algorithm 2)
+# ---------------------------------------------------------------------------------------
+
+def _policy_reference(tile_max_raw, sigma, T):
+    """The shifting maximum per tile, recomputed from the tile maxima alone in float32."""
+    f = np.float32
+    used = f(-np.inf)
+    out = []
+    for t in tile_max_raw:
+        cand = max(used, f(t))
+        if used == -np.inf or not T > 0:
+            used = cand
+        elif f(f(f(sigma) * cand) - f(f(sigma) * used)) > f(T):
+            used = cand
+        out.append(f(f(sigma) * used))
+    return np.array(out, np.float32)
+
+
+@pytest.mark.parametrize("T", [0.0, 0.75, 3.0, 1e9])
+def test_threshold_policy_of_the_shifting_maximum(oracle, T):
+    rng = np.random.default_rng(21)
+    sigma = float(np.float32(0.125))
+    raw = (rng.normal(0, 12, (16, 1024)) + np.linspace(0, 40, 1024)[None, :]).astype(np.float32)  # maxima keep growing
+    raw[3, :200] = -np.inf
+    codes, scales, ms = oracle.online_codes(raw, 128, sigma, *MEAN, rescale_threshold=T)
+    c0, s0, ms0 = oracle.online_codes(raw, 128, sigma, *MEAN)
+    tile_max = raw.reshape(16, 8, 128).max(-1)
+    for i in range(16):
+        assert np.array_equal(ms[i], _policy_reference(tile_max[i], sigma, T))
+    if T == 0.0:
+        assert np.array_equal(codes, c0) and np.array_equal(scales, s0) and np.array_equal(ms, ms0)
+    else:
+        with np.errstate(invalid="ignore"):
+            assert np.all((ms <= ms0) | np.isnan(ms0 - ms))          # never above the true running maximum
+            gap = ms0 - ms
+        assert np.nanmax(gap) <= T * (1 + 1e-6) + 1e-6               # and at most T below it
+        assert (np.diff(ms, axis=1) != 0).sum() < (np.diff(ms0, axis=1) != 0).sum() or T < 1.0
+    if T >= 1e9:
+        assert np.all(ms[:, 1:] == ms[:, :1]) or np.isinf(ms[3, 0])   # the first finite maximum is kept for good
+
+
+def test_threshold_policy_codes_are_the_stage_codes_for_the_kept_maximum(oracle):
+    """Per tile, the operand equals the standalone stage run with row_max = the kept maximum: the policy changes
+    which maximum shifts the scores and nothing else; shifted scores above zero only raise the block exponents."""
+    rng = np.random.default_rng(22)
+    sigma = float(np.float32(0.2))
+    raw = (rng.normal(0, 8, (8, 512)) + np.linspace(0, 25, 512)[None, :]).astype(np.float32)
+    codes, scales, ms = oracle.online_codes(raw, 128, sigma, *MEAN, rescale_threshold=2.5)
+    assert scales.max() > 124                                          # some block maximum sits above the kept maximum
+    for j in range(4):
+        tile = np.ascontiguousarray(raw[:, 128 * j:128 * (j + 1)])
+        c, s = oracle.probgen(tile, ms[:, j].copy(), sigma, *MEAN)
+        assert np.array_equal(c, codes[:, 64 * j:64 * (j + 1)]) and np.array_equal(s, scales[:, 4 * j:4 * (j + 1)])
+    # shift-equivariance: against threshold 0 the codes agree wherever the two maxima differ by a multiple of
+    # ln 2 ... in general they differ, but the represented probabilities relative to the same reference agree
+    c0, s0, ms0 = oracle.online_codes(raw, 128, sigma, *MEAN)
+    p = efq_math.C8[oracle.unpack_codes(codes)] * np.repeat(np.exp2(scales.astype(float) - 127), 32, 1) * \
+        np.repeat(np.exp(ms.astype(float)), 128, 1)
+    p0 = efq_math.C8[oracle.unpack_codes(c0)] * np.repeat(np.exp2(s0.astype(float) - 127), 32, 1) * \
+        np.repeat(np.exp(ms0.astype(float)), 128, 1)
+    big = p0 > 1e-3 * p0.max(axis=1, keepdims=True)
+    both = big & (p > 0)
+    assert both.sum() > 0.9 * big.sum()                                 # the smallest code may fall to zero, rarely
+    assert np.all(np.abs(np.log(p[both] / p0[both])) < 0.75)            # same value up to one code step
+
+
+@pytest.mark.parametrize("path", ["efq", "etq", "efq_lut"])
+def test_threshold_policy_leaves_the_attention_output_in_the_same_error_band(oracle, path):
+    case, q, k, v, rows = _small_case(S=384)
+    ex = oracle.attention_rows(q, k, v, rows, True, case.softmax_scale, "exact")
+    o0 = oracle.attention_rows(q, k, v, rows, True, case.softmax_scale, path)
+    oT = oracle.attention_rows(q, k, v, rows, True, case.softmax_scale, path, rescale_threshold=4.0)
+    e0 = np.linalg.norm(o0 - ex) / np.linalg.norm(ex)
+    eT = np.linalg.norm(oT - ex) / np.linalg.norm(ex)
+    assert abs(eT - e0) < 0.25 * e0
+    assert np.linalg.norm(oT - o0) / np.linalg.norm(o0) < e0
