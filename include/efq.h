@@ -47,7 +47,7 @@ typedef enum {
  * (Eq. d8-index).  (tau, h) are global, fixed after calibration; the operating points
  * printed in the paper are EFQ-Mean (-3.06, 2.30), EFQ-MMLU (-2.90, 2.00) and
  * EFQ-Balance (-2.10, 2.70).  Passing NULL for a params pointer selects EFQ-Mean,
- * variant 0, kv_tile 128. */
+ * variant 0, kv_tile 128, rescale_threshold 0. */
 typedef struct {
     float tau;
     float h;          /* > 0 */
@@ -61,6 +61,14 @@ typedef struct {
     int32_t kv_tile;  /* Bc, keys per online-softmax step; 0 = default (128).  The shifted score uses the
                          running row maximum that includes the current KV block (Algorithm 2, steps 2-3),
                          so codes depend on this width.  Must be 128 in this build. */
+    float rescale_threshold; /* T >= 0 in scaled-score units.  0 (default) is Algorithm 2 as printed: the running
+                         maximum shifts the scores and the history is rescaled whenever it grows.  T > 0 (not in
+                         the paper) keeps the shifting maximum m from tile to tile while the true running maximum
+                         exceeds it by at most T: with cand = max(m, tile maximum), m <- cand if m = -inf or
+                         fl(fl(scale cand) - fl(scale m)) > T, else m stays; a tile that keeps m needs no
+                         rescaling of the accumulators.  Shifted scores may then reach +T; the scale rule is
+                         shift-equivariant, so only block exponents move - but codes differ from T = 0.  Used by
+                         the fused forwards only (efq_probgen takes its row maximum from the caller). */
 } efq_params_t;
 
 /* Optional debug dump of the fused forward for one head and a range of query rows.

@@ -30,7 +30,8 @@ EXPORTS = ["efq_probgen", "exp_then_quantize_probgen", "efq_attention_workspace_
 
 
 class EfqParams(C.Structure):
-    _fields_ = [("tau", C.c_float), ("h", C.c_float), ("variant", C.c_int32), ("kv_tile", C.c_int32)]
+    _fields_ = [("tau", C.c_float), ("h", C.c_float), ("variant", C.c_int32), ("kv_tile", C.c_int32),
+                ("rescale_threshold", C.c_float)]
 
 
 class EfqDebug(C.Structure):
@@ -125,7 +126,8 @@ def _params(params) -> Optional[EfqParams]:
     tau, h = params[0], params[1]
     variant = params[2] if len(params) > 2 else 0
     kv_tile = params[3] if len(params) > 3 else 0
-    return EfqParams(float(tau), float(h), int(variant), int(kv_tile))
+    threshold = params[4] if len(params) > 4 else 0.0
+    return EfqParams(float(tau), float(h), int(variant), int(kv_tile), float(threshold))
 
 
 def _ptr(t) -> Optional[int]:

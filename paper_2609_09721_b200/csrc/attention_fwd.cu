@@ -97,6 +97,7 @@ struct FwdParams {
     efq_debug_t dbg;
     int has_dbg;
     int inject_skip_loads;    // test hook: the TMA thread loads Q only, so the first wait on K/V runs out
+    float rescale_threshold;  // 0: Algorithm 2; > 0: the shifting maximum is kept while the true one is at most this far above
 };
 
 // Bounded wait of one thread.  Returns false on timeout (recorded in the status word) or CTA-wide abort.
@@ -394,7 +395,11 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 if (!have_prev && !wait_all(&sm->x_bar[sb ^ 1][quarter], static_cast<uint32_t>(((j - 1) >> 1) & 1), sm, P.status)) { ok = false; break; }
                 m_prev = sm->runmax[sb ^ 1][row];
             }
-            const float m_new = fmaxf(fmaxf(m_prev, bmax[0]), max3(bmax[1], bmax[2], bmax[3]));
+            float m_new = fmaxf(fmaxf(m_prev, bmax[0]), max3(bmax[1], bmax[2], bmax[3]));
+            if (P.rescale_threshold > 0.0f && m_prev != -INFINITY) {      // optional policy: keep the old maximum
+                const float ahead = __fsub_rn(__fmul_rn(K.sigma, m_new), __fmul_rn(K.sigma, m_prev));
+                if (!(ahead > P.rescale_threshold)) m_new = m_prev;
+            }
             sm->runmax[sb][row] = m_new;
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&sm->x_bar[sb][quarter]);
@@ -576,7 +581,7 @@ cudaError_t launch_main(bool debug, bool fix8, dim3 grid, size_t smem, cudaStrea
 efq_status_t attention_impl(const void* q, const void* k, const void* v, float* o, int B, int Hq, int Hkv, int64_t Sq,
                             int64_t Sk, int d, int causal, float softmax_scale, int producer, float tau, float h,
                             void* workspace, size_t workspace_bytes, const efq_debug_t* debug, cudaStream_t stream,
-                            bool do_quantize, bool do_forward, bool inject_skip_loads = false)
+                            bool do_quantize, bool do_forward, bool inject_skip_loads = false, float rescale_threshold = 0.0f)
 {
     if (!q || !k || !v || !o) return EFQ_ERR_INVALID_ARG;
     if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0 || Hq % Hkv != 0) return EFQ_ERR_INVALID_ARG;
@@ -617,6 +622,7 @@ efq_status_t attention_impl(const void* q, const void* k, const void* v, float* 
     P.o = o;
     P.status = reinterpret_cast<uint32_t*>(ws + w.status);
     P.inject_skip_loads = inject_skip_loads ? 1 : 0;
+    P.rescale_threshold = rescale_threshold;
     P.has_dbg = debug ? 1 : 0;
     if (debug) P.dbg = *debug; else P.dbg = efq_debug_t{};
 
@@ -647,15 +653,18 @@ extern "C" size_t efq_attention_workspace_bytes(int B, int Hq, int Hkv, int64_t 
 }
 
 // Producer ids inside the library: 0 = EFQ (affine rule), 1 / 2 = exp-then-quantize scale4 / scale6, 3 = EFQ-LUT.
-static bool read_params(const efq_params_t* params, float& tau, float& h, bool& lut, efq_status_t& st)
+static bool read_params(const efq_params_t* params, float& tau, float& h, bool& lut, float& threshold, efq_status_t& st)
 {
     tau = -3.06f;
     h = 2.30f;
     lut = false;
+    threshold = 0.0f;
     st = EFQ_OK;
     if (params) {
         if (params->variant != 0 && params->variant != 1) { st = EFQ_ERR_UNSUPPORTED; return false; }
         if (params->kv_tile != 0 && params->kv_tile != 128) { st = EFQ_ERR_UNSUPPORTED; return false; }
+        if (!(params->rescale_threshold >= 0.0f)) { st = EFQ_ERR_INVALID_ARG; return false; }   // negative or NaN
+        threshold = params->rescale_threshold;
         lut = params->variant == 1;
         if (!lut) {                 // the LUT variant has its own fixed (tau16, h16): tau and h are not read
             tau = params->tau;
@@ -670,12 +679,12 @@ extern "C" efq_status_t efq_attention_fwd(const void* q, const void* k, const vo
                                           const efq_params_t* params, void* workspace, size_t workspace_bytes,
                                           const efq_debug_t* debug, void* stream)
 {
-    float tau, h;
+    float tau, h, threshold;
     bool lut;
     efq_status_t st;
-    if (!read_params(params, tau, h, lut, st)) return st;
+    if (!read_params(params, tau, h, lut, threshold, st)) return st;
     return efq::attention_impl(q, k, v, o, B, Hq, Hkv, Sq, Sk, d, causal, softmax_scale, lut ? 3 : 0, tau, h, workspace,
-                               workspace_bytes, debug, static_cast<cudaStream_t>(stream), true, true);
+                               workspace_bytes, debug, static_cast<cudaStream_t>(stream), true, true, false, threshold);
 }
 
 extern "C" efq_status_t exp_then_quantize_attention_fwd(const void* q, const void* k, const void* v, float* o, int B,
@@ -710,14 +719,14 @@ extern "C" efq_status_t efq_attention_fwd_quantized(float* o, int B, int Hq, int
                                                     const efq_params_t* params, void* workspace, size_t workspace_bytes,
                                                     const efq_debug_t* debug, void* stream)
 {
-    float tau, h;
+    float tau, h, threshold;
     bool lut;
     efq_status_t st;
-    if (!read_params(params, tau, h, lut, st)) return st;
+    if (!read_params(params, tau, h, lut, threshold, st)) return st;
     if (producer == 0 && lut) producer = 3;
     const void* nz = reinterpret_cast<const void*>(16);   // operands already live in the workspace
     return efq::attention_impl(nz, nz, nz, o, B, Hq, Hkv, Sq, Sk, d, causal, softmax_scale, producer, tau, h, workspace,
-                               workspace_bytes, debug, static_cast<cudaStream_t>(stream), false, true);
+                               workspace_bytes, debug, static_cast<cudaStream_t>(stream), false, true, false, threshold);
 }
 
 extern "C" efq_status_t efq_attention_fwd_host(const void* q_host, const void* k_host, const void* v_host, float* o_host,
@@ -728,10 +737,10 @@ extern "C" efq_status_t efq_attention_fwd_host(const void* q_host, const void* k
 {
     if (!q_host || !k_host || !v_host || !o_host || !q_dev || !k_dev || !v_dev || !o_dev) return EFQ_ERR_INVALID_ARG;
     if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0) return EFQ_ERR_INVALID_ARG;
-    float tau, h;
+    float tau, h, threshold;
     bool lut;
     efq_status_t st;
-    if (!read_params(params, tau, h, lut, st)) return st;
+    if (!read_params(params, tau, h, lut, threshold, st)) return st;
     if (producer == 0 && lut) producer = 3;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t qb = static_cast<size_t>(B) * Hq * Sq * d * 2, kb = static_cast<size_t>(B) * Hkv * Sk * d * 2;
@@ -739,7 +748,7 @@ extern "C" efq_status_t efq_attention_fwd_host(const void* q_host, const void* k
     if (cudaMemcpyAsync(k_dev, k_host, kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return EFQ_ERR_CUDA;
     if (cudaMemcpyAsync(v_dev, v_host, kb, cudaMemcpyHostToDevice, s) != cudaSuccess) return EFQ_ERR_CUDA;
     st = efq::attention_impl(q_dev, k_dev, v_dev, o_dev, B, Hq, Hkv, Sq, Sk, d, causal, softmax_scale, producer, tau, h,
-                             workspace, workspace_bytes, nullptr, s, true, true);
+                             workspace, workspace_bytes, nullptr, s, true, true, false, threshold);
     if (st != EFQ_OK) return st;
     if (cudaMemcpyAsync(o_host, o_dev, static_cast<size_t>(B) * Hq * Sq * d * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess)
         return EFQ_ERR_CUDA;
@@ -791,10 +800,10 @@ extern "C" efq_status_t efq_attention_fwd_static(const void* q, const void* k, c
                                                  int Hkv, int64_t Sq, int64_t Sk, int d, int causal,
                                                  float softmax_scale, const efq_params_t* params, void* stream)
 {
-    float tau, h;
+    float tau, h, threshold;
     bool lut;
     efq_status_t st;
-    if (!read_params(params, tau, h, lut, st)) return st;
+    if (!read_params(params, tau, h, lut, threshold, st)) return st;
     if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0) return EFQ_ERR_INVALID_ARG;
     if (d != 128) return EFQ_ERR_UNSUPPORTED;
     const size_t need = efq_attention_workspace_bytes(B, Hq, Hkv, Sq, Sk, d);
@@ -804,5 +813,5 @@ extern "C" efq_status_t efq_attention_fwd_static(const void* q, const void* k, c
     st = static_scratch_for_current_device(&scratch);
     if (st != EFQ_OK) return st;
     return efq::attention_impl(q, k, v, o, B, Hq, Hkv, Sq, Sk, d, causal, softmax_scale, lut ? 3 : 0, tau, h, scratch,
-                               EFQ_STATIC_SCRATCH_BYTES, nullptr, static_cast<cudaStream_t>(stream), true, true);
+                               EFQ_STATIC_SCRATCH_BYTES, nullptr, static_cast<cudaStream_t>(stream), true, true, false, threshold);
 }

@@ -228,6 +228,7 @@ extern "C" efq_status_t efq_calibrate(const void* q, const void* k, const void* 
             p.h = hs[ih];
             p.variant = 0;
             p.kv_tile = 0;
+            p.rescale_threshold = 0.0f;
             st = efq_attention_fwd_quantized(o_tmp, B, Hq, Hkv, Sq, Sk, d, causal, softmax_scale, 0, &p, workspace,
                                              workspace_bytes, nullptr, stream);
             if (st != EFQ_OK) return st;

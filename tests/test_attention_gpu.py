@@ -36,7 +36,7 @@ def _visible(case, i):
     return min(case.Sk, i + case.Sk - case.Sq + 1) if case.causal else case.Sk
 
 
-def _check_dump(oracle, case, dump, rows, params, producer="efq", want=None):
+def _check_dump(oracle, case, dump, rows, params, producer="efq", want=None, threshold=0.0):
     """L1: operand bit-exact on the kernel's own scores; raw scores equal to the oracle's."""
     raw = dump.raw_scores.cpu().numpy()
     codes = dump.codes.cpu().numpy()
@@ -46,7 +46,8 @@ def _check_dump(oracle, case, dump, rows, params, producer="efq", want=None):
         nv = _visible(case, int(i))
         assert np.all(np.isfinite(raw[n, :nv])), "visible scores must be written"
         raw[n, nv:] = -np.inf
-    oc, osc, oms = oracle.online_codes(raw, 128, case.softmax_scale, *params, producer=producer)
+    oc, osc, oms = oracle.online_codes(raw, 128, case.softmax_scale, *params, producer=producer,
+                                       rescale_threshold=threshold)
     for n, (_, _, i) in enumerate(rows):
         nt = (_visible(case, int(i)) + 127) // 128
         assert np.array_equal(ms[n, :nt], oms[n, :nt])
@@ -147,6 +148,40 @@ def test_lut_variant_fused_forward(oracle, S, Hq, Hkv, causal):
     torch.cuda.synchronize()
     if S >= 384:
         assert not torch.equal(o, o3)
+
+
+@pytest.mark.parametrize("S,Hq,Hkv,causal,T,variant", [(1024, 1, 1, False, 2.0, 0), (640, 2, 1, True, 0.5, 0),
+                                                       (1000, 2, 2, True, 6.0, 0), (512, 1, 1, True, 3.0, 1)])
+def test_thresholded_rescaling_policy(oracle, S, Hq, Hkv, causal, T, variant):
+    """rescale_threshold > 0 (not in the paper): the kept maximum, the operand and O follow the oracle's model of
+    the policy; K outliers make the running maximum move."""
+    case = inputs.AttentionCase("thr", 1, Hq, Hkv, S, S, 128, causal, 70 + S, "k_outliers")
+    (q, k, v), (dq, dk, dv) = _case_tensors(case)
+    head = Hq - 1
+    dump = binding.DebugDump(0, head, 0, S, S)
+    params = (MEAN[0], MEAN[1], variant, 0, T)
+    o = binding.efq_attention_fwd(dq, dk, dv, causal, 0.0, params, debug=dump)
+    torch.cuda.synchronize()
+    path = "efq_lut" if variant else "efq"
+    rows = np.array([(0, h, i) for h in range(Hq) for i in range(S)], np.int64)
+    want_o = oracle.attention_rows(q, k, v, rows, causal, case.softmax_scale, path, rescale_threshold=T)
+    got = o.cpu().numpy().reshape(-1, 128)
+    assert np.abs(got - want_o).max() <= TOL_O
+    _check_dump(oracle, case, dump, _all_rows(case, head, 0, S), MEAN, producer=path, threshold=T)
+    # the policy is in force: the kept maximum differs from the running maximum somewhere, and with it the output
+    o0 = binding.efq_attention_fwd(dq, dk, dv, causal, 0.0, (MEAN[0], MEAN[1], variant))
+    torch.cuda.synchronize()
+    assert not torch.equal(o, o0)
+    o2 = binding.efq_attention_fwd(dq, dk, dv, causal, 0.0, params)          # production instantiation
+    torch.cuda.synchronize()
+    assert torch.equal(o, o2)
+
+
+def test_negative_threshold_is_refused():
+    q = torch.zeros((1, 1, 128, 128), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(binding.EfqError) as e:
+        binding.efq_attention_fwd(q, q, q, params=(-3.06, 2.30, 0, 0, -1.0))
+    assert e.value.status == 1
 
 
 @pytest.mark.parametrize("mode,path", [(0, "etq"), (1, "etq6")])
