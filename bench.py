@@ -50,6 +50,8 @@ def workload_case(name: str) -> inputs.AttentionCase:
         return inputs.case_wan22(32760, seed=5)
     if name == "single_head_1024":
         return inputs.case_single_head(1024, seed=1)
+    if name == "wan22_4096":    # small non-causal case (24 heads, 32 KV tiles per CTA) for full-set profiler captures
+        return inputs.case_wan22(4096, seed=5)
     if name == "qwen3_8b_2k":   # small case for smoke runs and profiler captures
         return inputs.case_qwen3_8b(2048, seed=3)
     raise SystemExit(f"unknown workload {name}")

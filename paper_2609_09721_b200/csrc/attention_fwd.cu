@@ -70,14 +70,14 @@ struct __align__(1024) Smem {
     uint8_t sf_p[2][kSfBytes];
     uint8_t sf_ones[kSfBytes];
     float runmax[2][kTile];   // running row maximum after the group's latest tile, raw score units
-    float alpha[2][kTile];    // rescale factor of the group's current tile, per row (1 where the maximum did not grow)
+    float alpha[4][kTile];    // [tile mod 4]: rescale factor of the tile, per row (1 where the maximum did not grow)
     uint64_t q_full;
     uint64_t k_full[kStages], k_empty[kStages];
     uint64_t v_full[kStages], v_empty[kStages];
     uint64_t s_full[2], s_empty[2];
     uint64_t p_full[2], p_empty[2];
     uint64_t x_bar[2][4];     // [group][lane quarter]: runmax of the group's latest tile is published
-    uint64_t a_bar[2][4];     // [group][lane quarter]: alpha of the group's current tile is published
+    uint64_t a_bar[4][4];     // [tile mod 4][lane quarter]: alpha of that tile is published
     uint64_t o_ready[2];      // accumulator rows rescaled (or found unchanged) for the tile of this parity
     uint64_t o_done;          // the last P~V of the work item has completed
     uint32_t tmem_base;
@@ -178,11 +178,10 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             ptx::mbar_init(&sm->p_full[i], kGroupWarps);
             ptx::mbar_init(&sm->p_empty[i], 1);
             ptx::mbar_init(&sm->o_ready[i], 4);
-            for (int qd = 0; qd < 4; ++qd) {
-                ptx::mbar_init(&sm->x_bar[i][qd], 1);
-                ptx::mbar_init(&sm->a_bar[i][qd], 1);
-            }
+            for (int qd = 0; qd < 4; ++qd) ptx::mbar_init(&sm->x_bar[i][qd], 1);
         }
+        for (int i = 0; i < 4; ++i)
+            for (int qd = 0; qd < 4; ++qd) ptx::mbar_init(&sm->a_bar[i][qd], 1);
         sm->abort_flag = (*reinterpret_cast<volatile uint32_t*>(P.status) != 0u) ? 1u : 0u;
         ptx::mbar_init_fence();
     }
@@ -303,9 +302,9 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         for (int64_t j = 0; j < n_tiles; ++j) {
             const int sb = static_cast<int>(j & 1);
             // every tile, so that each phase of this barrier is seen in order
-            if (!wait_all(&sm->a_bar[sb][quarter], static_cast<uint32_t>((j >> 1) & 1), sm, P.status)) break;
+            if (!wait_all(&sm->a_bar[j & 3][quarter], static_cast<uint32_t>((j >> 2) & 1), sm, P.status)) break;
             if (j > 0) {
-                const float alpha = sm->alpha[sb][row];
+                const float alpha = sm->alpha[j & 3][row];
                 const bool any = __any_sync(0xffffffffu, alpha != 1.0f);
                 // every tile, so that each phase of this barrier is seen in order
                 if (!wait_all(&sm->p_empty[sb ^ 1], static_cast<uint32_t>(((j - 1) >> 1) & 1), sm, P.status)) break;
@@ -400,19 +399,20 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 const float ahead = __fsub_rn(__fmul_rn(K.sigma, m_new), __fmul_rn(K.sigma, m_prev));
                 if (!(ahead > P.rescale_threshold)) m_new = m_prev;
             }
-            sm->runmax[sb][row] = m_new;
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&sm->x_bar[sb][quarter]);
             const float m_s_prev = __fmul_rn(K.sigma, m_prev);
             const float m_s = __fmul_rn(K.sigma, m_new);
             const bool grew = m_new > m_prev && m_prev != -INFINITY;      // history exists and must be rescaled
             const float alpha = grew ? ex2_approx(__fmul_rn(__fsub_rn(m_s_prev, m_s), K.LOG2E)) : 1.0f;
-
-            // P~V of tile j-2 finished: the P buffer is free, and so is alpha[sb] (its reader ran before that P~V)
-            if (!have_p && !wait_all(&sm->p_empty[sb], ph2 ^ 1u, sm, P.status)) { ok = false; break; }
-            sm->alpha[sb][row] = alpha;
+            // One publication for both readers: the running maximum for the other group, alpha for the rescaling
+            // warps.  alpha sits in a ring of four tiles: slot j mod 4 was last read for tile j-4, before P~V_{j-4}
+            // was released, and this group waited for the end of P~V_{j-4} before it stored the codes of tile j-2.
+            sm->runmax[sb][row] = m_new;
+            sm->alpha[j & 3][row] = alpha;
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&sm->a_bar[sb][quarter]);
+            if (lane == 0) {
+                ptx::mbar_arrive(&sm->x_bar[sb][quarter]);
+                ptx::mbar_arrive(&sm->a_bar[j & 3][quarter]);
+            }
 
             // ---- probability operand (Algorithm 1 per block): codes and scales straight into the MMA operand
             uint32_t sfword = 0;
@@ -421,6 +421,9 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 uint4 codes;
                 uint32_t byte;
                 produce32<PRODUCER, FIX8>(&r[g * 32], bmax[g], m_s, K, codes, byte);
+                if (g == 0 && !have_p) {      // P~V of tile j-2 must have finished: it reads the group's P buffer
+                    if (!wait_all(&sm->p_empty[sb], ph2 ^ 1u, sm, P.status)) { ok = false; break; }
+                }
                 *reinterpret_cast<uint4*>(sm->p[sb] + p_swizzled_offset(row, g)) = codes;
                 sfword |= byte << (8 * g);
                 if (DEBUG && dbg_row) {
@@ -431,6 +434,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                     }
                 }
             }
+            if (!ok) break;               // the bounded wait inside the block loop gave up
             *reinterpret_cast<uint32_t*>(sm->sf_p[sb] + (row & 31u) * 16u + (row >> 5) * 4u) = sfword;
             if (DEBUG && dbg_row) {
                 if (P.dbg.raw_scores) {
