@@ -354,13 +354,14 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const int64_t nblk_all = (P.Sk + 31) / 32;
         const int64_t ntile_all = (P.Sk + kTile - 1) / kTile;
         bool ok = true;
+        bool s_ready = false;             // answer of a poll of s_full for this tile, asked at the end of the previous one
 
         for (int64_t j = group; j < n_tiles; j += 2) {
             const int sb = group;                                         // S, P and exchange buffers belong to the group
             const uint32_t ph2 = static_cast<uint32_t>((j >> 1) & 1);
 
             // ---- scores of tile j: TMEM -> registers (Algorithm 2, step 1 happened on the tensor core)
-            if (!wait_all(&sm->s_full[sb], ph2, sm, P.status)) { ok = false; break; }
+            if (!s_ready && !wait_all(&sm->s_full[sb], ph2, sm, P.status)) { ok = false; break; }
             ptx::tc_fence_after_sync();
             float r[128];
             float bmax[4];
@@ -375,9 +376,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 have_prev = j == 0 || ptx::mbar_try_wait(&sm->x_bar[sb ^ 1][quarter], static_cast<uint32_t>(((j - 1) >> 1) & 1));
                 have_p = ptx::mbar_try_wait(&sm->p_empty[sb], ph2 ^ 1u);
                 ptx::tmem_wait_ld();
-                ptx::tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&sm->s_empty[sb]);
+                ptx::tc_fence_before_sync();          // the S buffer is handed back with the joint publication below
                 const int64_t key0 = j * kTile;
                 if (key0 + 127 > limit) {     // diagonal or ragged tile: keys past the row's limit are masked in place
 #pragma unroll
@@ -412,6 +411,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             if (lane == 0) {
                 ptx::mbar_arrive(&sm->x_bar[sb][quarter]);
                 ptx::mbar_arrive(&sm->a_bar[j & 3][quarter]);
+                ptx::mbar_arrive(&sm->s_empty[sb]);           // every lane's scores are in registers (wait::ld above)
             }
 
             // ---- probability operand (Algorithm 1 per block): codes and scales straight into the MMA operand
@@ -444,6 +444,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 if (P.dbg.row_max) P.dbg.row_max[drow * ntile_all + j] = m_s;
             }
 
+            s_ready = j + 2 < n_tiles && ptx::mbar_try_wait(&sm->s_full[sb], ph2 ^ 1u);
             ptx::fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&sm->p_full[sb]);
