@@ -365,7 +365,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             ptx::tc_fence_after_sync();
             float r[128];
             float bmax[4];
-            bool have_prev, have_p;
+            bool have_prev;
             {
                 const uint32_t s_addr = tmem + lane_base + kColS + 128 * sb;
                 ptx::tmem_ld32f<0>(s_addr, r);
@@ -374,7 +374,6 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 ptx::tmem_ld32f<96>(s_addr + 96, r);
                 // polls whose answers are needed later travel while the scores do
                 have_prev = j == 0 || ptx::mbar_try_wait(&sm->x_bar[sb ^ 1][quarter], static_cast<uint32_t>(((j - 1) >> 1) & 1));
-                have_p = ptx::mbar_try_wait(&sm->p_empty[sb], ph2 ^ 1u);
                 ptx::tmem_wait_ld();
                 ptx::tc_fence_before_sync();          // the S buffer is handed back with the joint publication below
                 const int64_t key0 = j * kTile;
@@ -413,6 +412,8 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 ptx::mbar_arrive(&sm->a_bar[j & 3][quarter]);
                 ptx::mbar_arrive(&sm->s_empty[sb]);           // every lane's scores are in registers (wait::ld above)
             }
+            // P~V of tile j-2 reads the group's P buffer: asked here, answered while block 0 is computed
+            const bool have_p = ptx::mbar_try_wait(&sm->p_empty[sb], ph2 ^ 1u);
 
             // ---- probability operand (Algorithm 1 per block): codes and scales straight into the MMA operand
             uint32_t sfword = 0;
