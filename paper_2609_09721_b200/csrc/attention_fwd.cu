@@ -354,24 +354,26 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const int64_t nblk_all = (P.Sk + 31) / 32;
         const int64_t ntile_all = (P.Sk + kTile - 1) / kTile;
         bool ok = true;
-        bool s_ready = false;             // answer of a poll of s_full for this tile, asked at the end of the previous one
+        bool in_flight = false;           // the scores of this tile were asked for at the end of the group's previous tile
+        float r[128];
+        const uint32_t s_addr = tmem + lane_base + kColS + 128 * group;
 
         for (int64_t j = group; j < n_tiles; j += 2) {
             const int sb = group;                                         // S, P and exchange buffers belong to the group
             const uint32_t ph2 = static_cast<uint32_t>((j >> 1) & 1);
 
             // ---- scores of tile j: TMEM -> registers (Algorithm 2, step 1 happened on the tensor core)
-            if (!s_ready && !wait_all(&sm->s_full[sb], ph2, sm, P.status)) { ok = false; break; }
-            ptx::tc_fence_after_sync();
-            float r[128];
-            float bmax[4];
-            bool have_prev;
-            {
-                const uint32_t s_addr = tmem + lane_base + kColS + 128 * sb;
+            if (!in_flight) {
+                if (!wait_all(&sm->s_full[sb], ph2, sm, P.status)) { ok = false; break; }
+                ptx::tc_fence_after_sync();
                 ptx::tmem_ld32f<0>(s_addr, r);
                 ptx::tmem_ld32f<32>(s_addr + 32, r);
                 ptx::tmem_ld32f<64>(s_addr + 64, r);
                 ptx::tmem_ld32f<96>(s_addr + 96, r);
+            }
+            float bmax[4];
+            bool have_prev;
+            {
                 // polls whose answers are needed later travel while the scores do
                 have_prev = j == 0 || ptx::mbar_try_wait(&sm->x_bar[sb ^ 1][quarter], static_cast<uint32_t>(((j - 1) >> 1) & 1));
                 ptx::tmem_wait_ld();
@@ -445,11 +447,21 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 if (P.dbg.row_max) P.dbg.row_max[drow * ntile_all + j] = m_s;
             }
 
-            s_ready = j + 2 < n_tiles && ptx::mbar_try_wait(&sm->s_full[sb], ph2 ^ 1u);
+            // The registers are free: if S of the group's next tile is there already (it is as a rule, S runs ahead),
+            // its scores set out now and travel while the operand is handed over and the loop turns.
+            in_flight = !DEBUG && j + 2 < n_tiles && ptx::mbar_try_wait(&sm->s_full[sb], ph2 ^ 1u);
+            if (in_flight) {
+                ptx::tc_fence_after_sync();
+                ptx::tmem_ld32f<0>(s_addr, r);
+                ptx::tmem_ld32f<32>(s_addr + 32, r);
+                ptx::tmem_ld32f<64>(s_addr + 64, r);
+                ptx::tmem_ld32f<96>(s_addr + 96, r);
+            }
             ptx::fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&sm->p_full[sb]);
         }
+        ptx::tmem_wait_ld();              // nothing may be in flight when a bounded wait gave up inside the loop
 
         // ---- final normalisation O = A / l: each group writes 64 of the 128 channels
         // (a barrier of its own: a group that skipped a phase of the other group's p_empty could not tell
