@@ -16,7 +16,9 @@
 //               Thread = query row: the 128 scores of the row come from TMEM straight into registers;
 //               block maxima, scale and codes are thread-local; codes go as 16-byte packed stores into
 //               the swizzled shared-memory A operand, the four scale bytes as one word into the scale
-//               tile.  No FP16/FP32 probability tile exists anywhere.
+//               tile.  No FP16/FP32 probability tile exists anywhere.  Per tile a warp publishes once (running
+//               maximum, alpha, hand-back of the S buffer), asks each barrier one step before it needs the
+//               answer, and sends for the scores of its next tile as soon as its registers are free.
 // The online recurrence is unchanged: when a row's maximum grows, the accumulator rows in TMEM
 // are rescaled by alpha = exp(m_old - m_new) before the next P~V MMA is released (warps 12-15).
 //
