@@ -230,6 +230,17 @@ def test_qwen3_8b_16k_full_size_sampled_rows(oracle):
     _sampled_parity(oracle, inputs.case_qwen3_8b(16384, seed=3), 256, "qwen3-8b S=16384")
 
 
+def test_wan22_32760_full_size_sampled_rows(oracle):
+    """WAN2.2-shaped configuration at full size (24 heads, S=32760 = 1023*32 + 24, non-causal): the launch
+    configuration the benchmark times, checked on sampled rows (first/last rows, tile edges, the ragged tail)."""
+    _sampled_parity(oracle, inputs.case_wan22(32760, seed=5), 96, "wan2.2 S=32760")
+
+
+def test_qwen3_8b_128k_full_size_sampled_rows(oracle):
+    """The long-context configuration at full size (32 q / 8 kv heads, S=131072, causal) on sampled rows."""
+    _sampled_parity(oracle, inputs.case_qwen3_8b(131072, seed=4), 48, "qwen3-8b S=131072")
+
+
 def test_attention_argument_errors():
     q = torch.zeros((1, 3, 128, 128), dtype=torch.bfloat16, device="cuda")
     k = torch.zeros((1, 2, 128, 128), dtype=torch.bfloat16, device="cuda")
