@@ -351,9 +351,31 @@ def run_cuda(args):
         binding.efq_attention_fwd_host(hq, hk, hv, ho, dq, dk, dv, o, case.causal, 0.0, 0, None, ws)
     e1.record(stream)
     barrier()
-    e2e_ms = max_over_ranks([e0.elapsed_time(e1) / e2e_steps], dev)[0]
+    e2e_plain_ms = max_over_ranks([e0.elapsed_time(e1) / e2e_steps], dev)[0]
     h2d = hq.numel() * 2 + hk.numel() * 2 + hv.numel() * 2
     d2h = ho.numel() * 4
+    # the same with the copies overlapped chunk by chunk (efq_attention_fwd_host_pipelined): every step still moves
+    # all inputs in and the whole output out; steps do not overlap one another (copy-in waits for the previous step)
+    s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    n_chunks = case.B * case.Hkv
+
+    def e2e_step():
+        s_in.wait_stream(stream)
+        binding.efq_attention_fwd_host_pipelined(hq, hk, hv, ho, dq, dk, dv, o, (s_in, stream, s_out), case.causal, 0.0, 0,
+                                                 None, ws, n_chunks)
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = max_over_ranks([e0.elapsed_time(e1) / e2e_steps], dev)[0]
+    if binding.efq_poll_status(ws) != 0:
+        raise SystemExit("bench.py: device status set after the end-to-end region")
 
     # standalone probability-generation stage (HBM-bound): EFQ vs exp-then-quantize, 4096 x 16384 fp32
     stage = None
@@ -460,7 +482,10 @@ def run_cuda(args):
                    "l2": "inputs larger than L2 (Q+K+V bf16 and fp32 O exceed 126 MB)", "parallelism": f"replicas x{world}"},
         "clocks": clocks,
         "e2e": {"value": whole_job_tflops(flops, e2e_ms, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms,
+                "api": "efq_attention_fwd_host_pipelined, %d chunks (KV heads), pinned host q/k/v in and fp32 o out every step" % n_chunks,
+                "single_stream_ms_per_step": e2e_plain_ms,
+                "single_stream_value": whole_job_tflops(flops, e2e_plain_ms, world)},
         "gpu_launches": 4 * args.steps,
         "roofline": {"kernel": "attention_fwd_kernel<EFQ>", "bound": "tensor", "achieved": main_tflops, "peak": fp4_peak,
                      "unit": "TFLOP/s", "frac": main_tflops / fp4_peak, "traffic": traffic,

@@ -162,6 +162,23 @@ efq_status_t efq_attention_fwd_host(const void* q_host, const void* k_host, cons
                                     const efq_params_t* params, void* workspace, size_t workspace_bytes,
                                     void* stream);
 
+/* efq_attention_fwd_host with the copies overlapped: the problem is cut into `n_chunks` runs of KV heads (with
+ * their query heads; a run never crosses a batch entry, so at most B * Hkv chunks are used), and chunk i+1's
+ * inputs travel on `stream_in` while chunk i is computed on `stream_compute` and chunk i-1's output travels on
+ * `stream_out` (three distinct streams; the host buffers should be pinned).  Same arithmetic and results as
+ * efq_attention_fwd_host: heads are independent.  All chunks share one workspace slot (they are computed in
+ * order): `workspace_bytes` must cover the workspace of one chunk plus 256 bytes, which the size for the whole
+ * problem does whenever two or more chunks are used (with a single chunk the call is efq_attention_fwd_host on
+ * `stream_compute`).  The call is asynchronous; when the work queued on
+ * `stream_compute` has completed, so have the last copies, and efq_poll_status(workspace, stream_compute) reports
+ * a device-side timeout of any chunk.  Errors as efq_attention_fwd_host, plus INVALID_ARG for n_chunks <= 0. */
+efq_status_t efq_attention_fwd_host_pipelined(const void* q_host, const void* k_host, const void* v_host, float* o_host,
+                                              void* q_dev, void* k_dev, void* v_dev, float* o_dev, int B, int Hq,
+                                              int Hkv, int64_t Sq, int64_t Sk, int d, int causal, float softmax_scale,
+                                              int producer, const efq_params_t* params, void* workspace,
+                                              size_t workspace_bytes, int n_chunks, void* stream_in,
+                                              void* stream_compute, void* stream_out);
+
 /* Built-in scratch of efq_attention_fwd_static, in bytes (4 MiB).  Enough for, e.g., one head of 8192 tokens or
  * 8 query / 2 KV heads of 2048 tokens; efq_attention_workspace_bytes() gives the need of a shape. */
 #define EFQ_STATIC_SCRATCH_BYTES (4u << 20)

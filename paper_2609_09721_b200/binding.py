@@ -23,7 +23,7 @@ STATIC_SCRATCH_BYTES = 4 << 20
 # every symbol include/efq.h declares
 EXPORTS = ["efq_probgen", "exp_then_quantize_probgen", "efq_attention_workspace_bytes", "efq_attention_fwd",
            "exp_then_quantize_attention_fwd", "efq_quantize_qkv", "efq_attention_fwd_quantized",
-           "efq_attention_fwd_host", "efq_attention_fwd_static", "efq_poll_status",
+           "efq_attention_fwd_host", "efq_attention_fwd_host_pipelined", "efq_attention_fwd_static", "efq_poll_status",
            "efq_exact_attention_fwd", "efq_relative_error", "efq_calibrate",
            "efq_fp4_mma_peak_probe", "efq_stage_microbench", "efq_attention_fwd_inject_timeout", "efq_status_string",
            "efq_version"]
@@ -78,6 +78,9 @@ def lib() -> C.CDLL:
         L.efq_attention_fwd_host.restype = i32
         L.efq_attention_fwd_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i64, i64, i32, i32, f32,
                                              i32, C.POINTER(EfqParams), vp, C.c_size_t, vp]
+        L.efq_attention_fwd_host_pipelined.restype = i32
+        L.efq_attention_fwd_host_pipelined.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i64, i64, i32, i32,
+                                                       f32, i32, C.POINTER(EfqParams), vp, C.c_size_t, i32, vp, vp, vp]
         L.efq_attention_fwd_static.restype = i32
         L.efq_attention_fwd_static.argtypes = [vp, vp, vp, vp, i32, i32, i32, i64, i64, i32, i32, f32,
                                                C.POINTER(EfqParams), vp]
@@ -272,6 +275,24 @@ def efq_attention_fwd_host(q_host, k_host, v_host, o_host, q_dev, k_dev, v_dev, 
                                       C.byref(p) if p is not None else None, workspace.data_ptr(),
                                       workspace.numel(), _stream(stream))
     _check(st, "efq_attention_fwd_host")
+    return o_host
+
+
+def efq_attention_fwd_host_pipelined(q_host, k_host, v_host, o_host, q_dev, k_dev, v_dev, o_dev, streams,
+                                     causal: bool = False, softmax_scale: float = 0.0, producer: int = 0, params=None,
+                                     workspace=None, n_chunks: int = 8):
+    """End-to-end form with the copies overlapped: ``streams`` = (copy-in, compute, copy-out) torch streams.
+    Synchronising the compute stream completes the call."""
+    B, Hq, Sq, d = q_host.shape
+    _, Hkv, Sk, _ = k_host.shape
+    assert not q_host.is_cuda and not o_host.is_cuda and q_dev.is_cuda and o_dev.is_cuda and len(streams) == 3
+    p = _params(params)
+    st = lib().efq_attention_fwd_host_pipelined(
+        q_host.data_ptr(), k_host.data_ptr(), v_host.data_ptr(), o_host.data_ptr(), q_dev.data_ptr(), k_dev.data_ptr(),
+        v_dev.data_ptr(), o_dev.data_ptr(), B, Hq, Hkv, Sq, Sk, d, int(bool(causal)), float(softmax_scale),
+        int(producer), C.byref(p) if p is not None else None, workspace.data_ptr(), workspace.numel(), int(n_chunks),
+        _stream(streams[0]), _stream(streams[1]), _stream(streams[2]))
+    _check(st, "efq_attention_fwd_host_pipelined")
     return o_host
 
 

@@ -775,6 +775,103 @@ extern "C" efq_status_t efq_attention_fwd_host(const void* q_host, const void* k
     return EFQ_OK;
 }
 
+namespace efq {
+namespace {
+// dst takes src's status if src reports one (keeps the first problem seen across the chunks of a pipelined call)
+__global__ void merge_status_kernel(uint32_t* dst, const uint32_t* src, int overwrite)
+{
+    const uint32_t v = *src;
+    if (overwrite || v != 0u) *dst = v;
+}
+}  // namespace
+}  // namespace efq
+
+extern "C" efq_status_t efq_attention_fwd_host_pipelined(const void* q_host, const void* k_host, const void* v_host,
+                                                         float* o_host, void* q_dev, void* k_dev, void* v_dev,
+                                                         float* o_dev, int B, int Hq, int Hkv, int64_t Sq, int64_t Sk,
+                                                         int d, int causal, float softmax_scale, int producer,
+                                                         const efq_params_t* params, void* workspace,
+                                                         size_t workspace_bytes, int n_chunks, void* stream_in,
+                                                         void* stream_compute, void* stream_out)
+{
+    if (!q_host || !k_host || !v_host || !o_host || !q_dev || !k_dev || !v_dev || !o_dev) return EFQ_ERR_INVALID_ARG;
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0 || Hq % Hkv != 0 || n_chunks <= 0) return EFQ_ERR_INVALID_ARG;
+    if (!workspace) return EFQ_ERR_WORKSPACE;
+    float tau, h, threshold;
+    bool lut;
+    efq_status_t st;
+    if (!read_params(params, tau, h, lut, threshold, st)) return st;
+    if (producer == 0 && lut) producer = 3;
+    cudaStream_t s_in = static_cast<cudaStream_t>(stream_in), s_c = static_cast<cudaStream_t>(stream_compute),
+                 s_out = static_cast<cudaStream_t>(stream_out);
+    // chunks are runs of KV heads inside one batch entry: contiguous slices of q, k, v and o
+    int per_batch = n_chunks / B;
+    if (per_batch < 1) per_batch = 1;
+    if (per_batch > Hkv) per_batch = Hkv;
+    const int heads_per_chunk = (Hkv + per_batch - 1) / per_batch;
+    const int group = Hq / Hkv;
+    if (B == 1 && heads_per_chunk >= Hkv)        // nothing to overlap: the plain form on the compute stream
+        return efq_attention_fwd_host(q_host, k_host, v_host, o_host, q_dev, k_dev, v_dev, o_dev, B, Hq, Hkv, Sq, Sk, d,
+                                      causal, softmax_scale, producer == 3 ? 0 : producer, params, workspace,
+                                      workspace_bytes, stream_compute);
+    if (!efq::shape_ok(1, heads_per_chunk * group, heads_per_chunk, Sq, Sk, d)) return EFQ_ERR_UNSUPPORTED;
+    const size_t slot = efq::plan_workspace(1, heads_per_chunk * group, heads_per_chunk, Sq, Sk).total;
+    if (workspace_bytes < slot + 256) return EFQ_ERR_WORKSPACE;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    uint32_t* agg = reinterpret_cast<uint32_t*>(ws + slot);          // first problem seen by any chunk
+    if (cudaMemsetAsync(agg, 0, 4, s_c) != cudaSuccess) return EFQ_ERR_CUDA;
+
+    const size_t q_head = static_cast<size_t>(Sq) * d * 2, kv_head = static_cast<size_t>(Sk) * d * 2;
+    const size_t o_head = static_cast<size_t>(Sq) * d * 4;
+    cudaEvent_t ev = nullptr;
+    auto fail = [&](efq_status_t code) { if (ev) cudaEventDestroy(ev); return code; };
+    for (int b = 0; b < B; ++b) {
+        for (int h0 = 0; h0 < Hkv; h0 += heads_per_chunk) {
+            const int nh = h0 + heads_per_chunk <= Hkv ? heads_per_chunk : Hkv - h0;
+            const size_t q_off = (static_cast<size_t>(b) * Hq + static_cast<size_t>(h0) * group) * q_head;
+            const size_t kv_off = (static_cast<size_t>(b) * Hkv + h0) * kv_head;
+            const size_t o_off = (static_cast<size_t>(b) * Hq + static_cast<size_t>(h0) * group) * o_head;
+            const uint8_t* qh = static_cast<const uint8_t*>(q_host) + q_off;
+            const uint8_t* kh = static_cast<const uint8_t*>(k_host) + kv_off;
+            const uint8_t* vh = static_cast<const uint8_t*>(v_host) + kv_off;
+            uint8_t* qd = static_cast<uint8_t*>(q_dev) + q_off;
+            uint8_t* kd = static_cast<uint8_t*>(k_dev) + kv_off;
+            uint8_t* vd = static_cast<uint8_t*>(v_dev) + kv_off;
+            uint8_t* od = reinterpret_cast<uint8_t*>(o_dev) + o_off;
+            // inputs of this chunk: stream_in
+            if (cudaMemcpyAsync(qd, qh, q_head * nh * group, cudaMemcpyHostToDevice, s_in) != cudaSuccess) return fail(EFQ_ERR_CUDA);
+            if (cudaMemcpyAsync(kd, kh, kv_head * nh, cudaMemcpyHostToDevice, s_in) != cudaSuccess) return fail(EFQ_ERR_CUDA);
+            if (cudaMemcpyAsync(vd, vh, kv_head * nh, cudaMemcpyHostToDevice, s_in) != cudaSuccess) return fail(EFQ_ERR_CUDA);
+            if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess) return EFQ_ERR_CUDA;
+            if (cudaEventRecord(ev, s_in) != cudaSuccess || cudaStreamWaitEvent(s_c, ev, 0) != cudaSuccess) return fail(EFQ_ERR_CUDA);
+            cudaEventDestroy(ev);     // released once the recorded work has completed
+            ev = nullptr;
+            // forward of this chunk: stream_compute (in order, so the one workspace slot is reused safely)
+            st = efq::attention_impl(qd, kd, vd, reinterpret_cast<float*>(od), 1, nh * group, nh, Sq, Sk, d, causal,
+                                     softmax_scale, producer, tau, h, ws, slot, nullptr, s_c, true, true, false, threshold);
+            if (st != EFQ_OK) return st;
+            efq::merge_status_kernel<<<1, 1, 0, s_c>>>(agg, reinterpret_cast<const uint32_t*>(ws), 0);
+            if (cudaGetLastError() != cudaSuccess) return EFQ_ERR_CUDA;
+            if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess) return EFQ_ERR_CUDA;
+            if (cudaEventRecord(ev, s_c) != cudaSuccess || cudaStreamWaitEvent(s_out, ev, 0) != cudaSuccess) return fail(EFQ_ERR_CUDA);
+            cudaEventDestroy(ev);
+            ev = nullptr;
+            // output of this chunk: stream_out
+            if (cudaMemcpyAsync(static_cast<uint8_t*>(static_cast<void*>(o_host)) + o_off, od, o_head * nh * group,
+                                cudaMemcpyDeviceToHost, s_out) != cudaSuccess)
+                return EFQ_ERR_CUDA;
+        }
+    }
+    // the status word efq_poll_status() reads takes the aggregate; stream_compute then waits for the last copies,
+    // so that synchronising stream_compute alone completes the call
+    efq::merge_status_kernel<<<1, 1, 0, s_c>>>(reinterpret_cast<uint32_t*>(ws), agg, 1);
+    if (cudaGetLastError() != cudaSuccess) return EFQ_ERR_CUDA;
+    if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess) return EFQ_ERR_CUDA;
+    if (cudaEventRecord(ev, s_out) != cudaSuccess || cudaStreamWaitEvent(s_c, ev, 0) != cudaSuccess) return fail(EFQ_ERR_CUDA);
+    cudaEventDestroy(ev);
+    return EFQ_OK;
+}
+
 extern "C" efq_status_t efq_poll_status(void* workspace, void* stream)
 {
     if (!workspace) return EFQ_ERR_INVALID_ARG;

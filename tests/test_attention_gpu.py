@@ -337,3 +337,28 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     torch.cuda.synchronize()
     want = binding.efq_attention_fwd(hq.cuda(), hk.cuda(), hv.cuda(), True)
     assert torch.equal(ho.cuda(), want)
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,S,chunks", [(1, 8, 4, 640, 4), (2, 4, 2, 384, 8), (1, 6, 3, 300, 2), (1, 2, 1, 256, 5)])
+def test_pipelined_host_entry_point_matches_device_entry_point(B, Hq, Hkv, S, chunks):
+    """Copies overlapped chunk by chunk over three streams: bit-identical to the one-shot forward."""
+    case = inputs.AttentionCase("hp", B, Hq, Hkv, S, S, 128, True, 77 + S, "k_outliers")
+    qb, kb, vb = inputs.make_qkv(case)
+    pin = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).pin_memory()
+    hq, hk, hv = pin(qb), pin(kb), pin(vb)
+    dq, dk, dv = torch.empty_like(hq, device="cuda"), torch.empty_like(hk, device="cuda"), torch.empty_like(hv, device="cuda")
+    do = torch.empty((B, Hq, S, 128), dtype=torch.float32, device="cuda")
+    ho = torch.zeros((B, Hq, S, 128), dtype=torch.float32).pin_memory()
+    ws = torch.empty(binding.efq_attention_workspace_bytes(B, Hq, Hkv, S, S, 128), dtype=torch.uint8, device="cuda")
+    streams = [torch.cuda.Stream() for _ in range(3)]
+    torch.cuda.synchronize()
+    for _ in range(2):      # twice: the workspace slot and the staging buffers are reused
+        binding.efq_attention_fwd_host_pipelined(hq, hk, hv, ho, dq, dk, dv, do, streams, True, 0.0, 0, None, ws, chunks)
+    streams[1].synchronize()          # the compute stream alone completes the call
+    assert binding.efq_poll_status(ws, streams[1]) == 0
+    want = binding.efq_attention_fwd(hq.cuda(), hk.cuda(), hv.cuda(), True)
+    torch.cuda.synchronize()
+    assert torch.equal(ho.cuda(), want)
+    with pytest.raises(binding.EfqError) as e:
+        binding.efq_attention_fwd_host_pipelined(hq, hk, hv, ho, dq, dk, dv, do, streams, True, 0.0, 0, None, ws, 0)
+    assert e.value.status == 1
