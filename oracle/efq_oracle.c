@@ -207,7 +207,10 @@ static efq_consts make_consts_lut(float sigma)
     return k;
 }
 
-/* producer ids: 0 = EFQ, 1 = exp-then-quantize scale4, 2 = exp-then-quantize scale6, 3 = EFQ-LUT */
+/* producer ids: 0 = EFQ, 1 = exp-then-quantize scale4, 2 = exp-then-quantize scale6, 3 = EFQ-LUT,
+ * 4 = exp-then-quantize scale4 whose DENOMINATOR is summed from the FP32 exponentials instead of the quantised
+ * operand (the convention of attention kernels that quantise P only for the P V product; reported as context,
+ * the paper's shared-operand rule is producers 0-3). */
 static efq_consts consts_for(int producer, float sigma, float tau, float h)
 {
     return producer == 3 ? make_consts_lut(sigma) : make_consts(sigma, tau, h);
@@ -374,14 +377,21 @@ static void online_row(const float* r, int64_t n_keys, const float* vhat, int d,
         for (int64_t t = t0; t < t1; t += MXB) {
             int n = t1 - t < MXB ? (int)(t1 - t) : MXB;
             uint8_t sb = is_efq(producer) ? efq_block(r + t, n, m_s, K, c)
-                                       : etq_block(r + t, n, m_s, K->sigma, producer - 1, c);
+                                       : etq_block(r + t, n, m_s, K->sigma, producer == 4 ? 0 : producer - 1, c);
             if (scales_out) scales_out[t / MXB] = sb;
             if (codes_out) pack_codes(c, n, codes_out + (t / MXB) * (MXB / 2));
             double s = ldexp(1.0, (int)sb - 127);
             for (int u = 0; u < n; ++u) {
                 double p = s * C8[c[u]]; /* p~_t = s_b * C8[c_t] */
-                if (p == 0.0) continue;
-                l += p;                                         /* Eq. denominator-basic */
+                if (producer == 4 && r[t + u] != -INFINITY) {   /* context variant: FP32 exponential in the denominator */
+                    float x = K->sigma * r[t + u];
+                    x = x - m_s;
+                    l += (double)(float)exp((double)x);
+                    if (p == 0.0) continue;
+                } else {
+                    if (p == 0.0) continue;
+                    l += p;                                     /* Eq. denominator-basic */
+                }
                 const float* vr = vhat + (t + u) * d;
                 for (int ch = 0; ch < d; ++ch) A[ch] += p * (double)vr[ch]; /* Eq. numerator-basic */
             }
@@ -427,7 +437,7 @@ static int64_t visible_keys(int64_t i, int64_t Sq, int64_t Sk, int causal)
 
 /* q [B,Hq,Sq,d], k, v [B,Hkv,Sk,d] as fp32 (exact widenings of the bf16 inputs).
  * rows [n_rows, 3] = (b, head, query index).  path: 0 = exact (double, unquantised),
- * 1 = EFQ, 2 = ETQ scale4, 3 = ETQ scale6, 4 = EFQ-LUT.  out [n_rows, d] fp32.
+ * 1 = EFQ, 2 = ETQ scale4, 3 = ETQ scale6, 4 = EFQ-LUT, 5 = ETQ scale4 with FP32 denominator.  out [n_rows, d] fp32.
  * Optional dumps (NULL to skip), each row-major over the sampled rows:
  *   raw [n_rows, Sk] (-inf where masked), codes [n_rows, nblk*16], scales [n_rows, nblk],
  *   ms [n_rows, ntile]. */

@@ -4,7 +4,8 @@ All arrays are numpy, host memory.  bf16 inputs are passed as float32 (exact wid
 Paths: "exact" (double softmax attention on the unquantised inputs), "efq" (Algorithm 2
 with Algorithm 1 as producer), "etq" (exp-then-quantize producer, block maximum scaled
 into [4, 8)), "etq6" (same with the block maximum scaled into (3, 6]), "efq_lut" (Algorithm 1 with
-the 16-level index and the folding table of the LUT variant; tau and h are not used).
+the 16-level index and the folding table of the LUT variant; tau and h are not used), "etq_fp32den"
+(attention_rows only: "etq" with the denominator summed from the FP32 exponentials; context, not the paper's rule).
 """
 from __future__ import annotations
 
@@ -16,7 +17,7 @@ from . import build as _build
 
 _lib = None
 
-PATHS = {"exact": 0, "efq": 1, "etq": 2, "etq6": 3, "efq_lut": 4}
+PATHS = {"exact": 0, "efq": 1, "etq": 2, "etq6": 3, "efq_lut": 4, "etq_fp32den": 5}
 PRODUCERS = {"efq": 0, "etq": 1, "etq6": 2, "efq_lut": 3}
 
 # (tau, h) operating points printed in the paper's "Parameter selection" paragraph.

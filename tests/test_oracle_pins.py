@@ -572,3 +572,20 @@ def test_threshold_policy_leaves_the_attention_output_in_the_same_error_band(ora
     eT = np.linalg.norm(oT - ex) / np.linalg.norm(ex)
     assert abs(eT - e0) < 0.25 * e0
     assert np.linalg.norm(oT - o0) / np.linalg.norm(o0) < e0
+
+
+def test_fp32_denominator_variant_of_the_baseline(oracle):
+    """Context variant: the quantised operand in the numerator, FP32 exponentials in the denominator.  With one KV
+    tile it is the closed form sum(p~ v^) / sum(exp(x)); against the shared-operand rule it differs by the ratio of
+    the two denominators, row by row."""
+    case, q, k, v, rows = _small_case(S=96)
+    sigma = case.softmax_scale
+    o_sh, d = oracle.attention_rows(q, k, v, rows, False, sigma, "etq", Bc=128, dumps=True)
+    o_fp = oracle.attention_rows(q, k, v, rows, False, sigma, "etq_fp32den", Bc=128)
+    codes = oracle.unpack_codes(d["codes"])[:, :96]
+    p_q = efq_math.C8[codes] * np.repeat(np.exp2(d["scales"].astype(float) - 127), 32, 1)[:, :96]
+    x = (np.float32(sigma) * d["raw"]).astype(np.float32) - d["ms"][:, :1]
+    p_f = np.exp(x.astype(np.float64)).astype(np.float32).astype(np.float64)
+    ratio = p_q.sum(1) / p_f.sum(1)
+    assert np.abs(o_fp - o_sh * ratio[:, None]).max() < 1e-5
+    assert np.abs(ratio - 1.0).max() < 0.2 and np.abs(ratio - 1.0).max() > 1e-4
