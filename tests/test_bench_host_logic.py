@@ -88,3 +88,10 @@ def test_clock_summary_keeps_only_samples_inside_the_timed_region():
     assert out["samples"] == 3 and out["power_w_max"] == 900.0
     empty = bench.summarize_clock_samples(samples, 20.0, 21.0, "nvml")
     assert empty["sm_mhz"] is None and "no samples" in empty["reasons"][0]
+
+
+def test_calibration_cli_grid_parsing():
+    from paper_2609_09721_b200 import calibrate
+    assert calibrate._grid("-3.6:-1.8:0.3") == [-3.6, -3.3, -3.0, -2.7, -2.4, -2.1, -1.8]
+    assert calibrate._grid("2:2:1") == [2.0]
+    assert set(calibrate.WORKLOADS) >= {"single_head_1024", "qwen3_8b_2k", "wan22_4096"}
