@@ -121,10 +121,9 @@ __device__ __forceinline__ void load8(const float* p, float (&r)[8])
 }
 
 template <int PRODUCER>
-__global__ void __launch_bounds__(kWarpsPerCta * 32)
-probgen_kernel(const float* __restrict__ scores, int64_t ld, const float* __restrict__ row_max,
-               int64_t rows, int64_t cols, ProducerConsts K, uint8_t* __restrict__ codes,
-               uint8_t* __restrict__ scales, int aligned32)
+__device__ __forceinline__ void probgen_body(const float* __restrict__ scores, int64_t ld, const float* __restrict__ row_max,
+                                             int64_t rows, int64_t cols, const ProducerConsts& K, uint8_t* __restrict__ codes,
+                                             uint8_t* __restrict__ scales, int aligned32)
 {
     const int lane = threadIdx.x & 31;
     const int64_t segs_per_row = (cols + kSegCols - 1) / kSegCols;
@@ -178,6 +177,23 @@ probgen_kernel(const float* __restrict__ scores, int64_t ld, const float* __rest
     }
 }
 
+template <int PRODUCER>
+__global__ void __launch_bounds__(kWarpsPerCta * 32)
+probgen_kernel(const float* __restrict__ scores, int64_t ld, const float* __restrict__ row_max, int64_t rows, int64_t cols,
+               ProducerConsts K, uint8_t* __restrict__ codes, uint8_t* __restrict__ scales, int aligned32)
+{
+    probgen_body<PRODUCER>(scores, ld, row_max, rows, cols, K, codes, scales, aligned32);
+}
+
+// The LUT producer is issue-bound and register-hungry (one code at a time through a 64-bit shift): it gains more from
+// three resident CTAs per SM than from the registers the compiler would otherwise take (69 -> 54 microseconds).
+__global__ void __launch_bounds__(kWarpsPerCta * 32, 3)
+probgen_lut_kernel(const float* __restrict__ scores, int64_t ld, const float* __restrict__ row_max, int64_t rows,
+                   int64_t cols, ProducerConsts K, uint8_t* __restrict__ codes, uint8_t* __restrict__ scales, int aligned32)
+{
+    probgen_body<kEfqLut>(scores, ld, row_max, rows, cols, K, codes, scales, aligned32);
+}
+
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 efq_status_t launch_probgen(int producer, const float* scores, int64_t ld, const float* row_max, int64_t rows,
@@ -208,7 +224,7 @@ efq_status_t launch_probgen(int producer, const float* scores, int64_t ld, const
         case kEfq:  probgen_kernel<kEfq><<<grid, block, 0, stream>>>(scores, ld, row_max, rows, cols, K, codes, scales, a32); break;
         case kEtq4: probgen_kernel<kEtq4><<<grid, block, 0, stream>>>(scores, ld, row_max, rows, cols, K, codes, scales, a32); break;
         case kEtq6: probgen_kernel<kEtq6><<<grid, block, 0, stream>>>(scores, ld, row_max, rows, cols, K, codes, scales, a32); break;
-        case kEfqLut: probgen_kernel<kEfqLut><<<grid, block, 0, stream>>>(scores, ld, row_max, rows, cols, K, codes, scales, a32); break;
+        case kEfqLut: probgen_lut_kernel<<<grid, block, 0, stream>>>(scores, ld, row_max, rows, cols, K, codes, scales, a32); break;
         default: return EFQ_ERR_INVALID_ARG;
     }
     return cudaGetLastError() == cudaSuccess ? EFQ_OK : EFQ_ERR_CUDA;
