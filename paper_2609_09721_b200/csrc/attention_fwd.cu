@@ -658,6 +658,7 @@ efq_status_t attention_impl(const void* q, const void* k, const void* v, float* 
         case 1: e = launch_main<1>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
         case 2: e = launch_main<2>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
         case 3: e = launch_main<3>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
+        case 4: e = launch_main<4>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
         default: return EFQ_ERR_INVALID_ARG;
     }
     return e == cudaSuccess ? EFQ_OK : EFQ_ERR_CUDA;
@@ -672,7 +673,8 @@ extern "C" size_t efq_attention_workspace_bytes(int B, int Hq, int Hkv, int64_t 
     return efq::plan_workspace(B, Hq, Hkv, Sq, Sk).total;
 }
 
-// Producer ids inside the library: 0 = EFQ (affine rule), 1 / 2 = exp-then-quantize scale4 / scale6, 3 = EFQ-LUT.
+// Producer ids inside the library: 0 = EFQ (affine rule), 1 / 2 = exp-then-quantize scale4 / scale6, 3 = EFQ-LUT,
+// 4 = exp-then-quantize scale4 with the scale folded into the exponential.
 static bool read_params(const efq_params_t* params, float& tau, float& h, bool& lut, float& threshold, efq_status_t& st)
 {
     tau = -3.06f;
@@ -712,8 +714,8 @@ extern "C" efq_status_t exp_then_quantize_attention_fwd(const void* q, const voi
                                                         float softmax_scale, int scale_mode, void* workspace,
                                                         size_t workspace_bytes, const efq_debug_t* debug, void* stream)
 {
-    if (scale_mode != 0 && scale_mode != 1) return EFQ_ERR_INVALID_ARG;
-    return efq::attention_impl(q, k, v, o, B, Hq, Hkv, Sq, Sk, d, causal, softmax_scale, 1 + scale_mode, 0.0f, 1.0f,
+    if (scale_mode < 0 || scale_mode > 2) return EFQ_ERR_INVALID_ARG;
+    return efq::attention_impl(q, k, v, o, B, Hq, Hkv, Sq, Sk, d, causal, softmax_scale, scale_mode == 2 ? 4 : 1 + scale_mode, 0.0f, 1.0f,
                                workspace, workspace_bytes, debug, static_cast<cudaStream_t>(stream), true, true);
 }
 

@@ -105,6 +105,36 @@ __device__ __forceinline__ uint32_t lut_code(float r, float A16, float B16)
     return static_cast<uint32_t>(kLutFold16 >> (4u * j)) & 15u;
 }
 
+// exp-then-quantize with the block scale folded into the exponential (the strongest form of the baseline on this
+// machine): p 2^-e = 2^(x log2(e) - e), so with t = fma(r, sigma log2(e), -m_s log2(e)) the scaled probability is one
+// FMA and one ex2 away from the raw score; the exponential is monotone, so the block maximum of p is ex2 of
+// t(rmax) and e = floor(t(rmax)) - 2 (block maximum in [4, 8)) needs no pass over p.  Same mathematics as
+// p = exp(x), e = floor(log2 max p) - 2, q = RNE(p 2^-e); rounding differs at knife-edges only.
+// The block's exponent is taken from x(rmax) = fl(fl(sigma rmax) - m_s), which is exactly 0 for the row maximum:
+// p = 1 sits on a power of two, and the fused form fma(rmax, c1, c0) lands a rounding error below it as often as
+// above, which would put the row's largest probability one binade too high and saturate it.
+struct FoldedScale {
+    float c1;       // sigma * log2(e)
+    float c0e;      // -m_s * log2(e) - e
+    uint32_t byte;  // e + 127, or 0 for a block without a finite score
+    bool live;
+};
+__device__ __forceinline__ FoldedScale etq_folded_scale(float rmax, float m_s, const ProducerConsts& K)
+{
+    FoldedScale f;
+    f.c1 = __fmul_rn(K.sigma, K.LOG2E);
+    const float c0 = __fmul_rn(-m_s, K.LOG2E);
+    f.live = rmax != -INFINITY;
+    float t = __fmul_rn(__fsub_rn(__fmul_rn(K.sigma, rmax), m_s), K.LOG2E);
+    t = fminf(fmaxf(t, -125.0f), 129.0f);            // e = floor(t) - 2 stays in [-127, 127]; NaN (no finite score) -> -125
+    float km;
+    asm("add.rm.f32 %0, %1, %2;" : "=f"(km) : "f"(t), "f"(12582912.0f));   // floor by a round-down add of 1.5 * 2^23
+    const float ef = __fsub_rn(__fsub_rn(km, 12582912.0f), 2.0f);
+    f.c0e = __fsub_rn(c0, ef);
+    f.byte = f.live ? (__float_as_uint(km) - 0x4B400000u - 2u + 127u) : 0u;
+    return f;
+}
+
 // Two floats -> one byte of E2M1 (round-to-nearest-even, saturating); `lo` lands in bits 0-3.
 __device__ __forceinline__ uint32_t cvt_e2m1x2(float lo, float hi)
 {

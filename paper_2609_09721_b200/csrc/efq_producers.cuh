@@ -38,7 +38,7 @@ __device__ __forceinline__ float block_max32(const float* r)
 
 // 32 scores of one microscaling block -> 16 bytes of codes + scale byte.
 // PRODUCER: 0 = EFQ (affine rule), 1 / 2 = exp-then-quantize with the block maximum in [4, 8) / (3, 6],
-// 3 = EFQ-LUT.
+// 3 = EFQ-LUT, 4 = exp-then-quantize [4, 8) with the scale folded into the exponential.
 //
 // EFQ (Algorithm 1), three FMA-pipe instructions per element, bit-identical to
 // c = floor(min(max(fma(r, A, Bb), 0), 7)):
@@ -87,6 +87,22 @@ __device__ __forceinline__ void produce32(const float* r, float rmax, float m_s,
 #pragma unroll
             for (int i = 0; i < 8; ++i) word |= lut_code(r[q * 8 + i], A16, B16) << (4 * i);
             w[q] = word;
+        }
+    } else if (PRODUCER == 4) {
+        // exp-then-quantize (block maximum in [4, 8)) with the scale folded into the exponential: one FMA, one ex2
+        // and half a conversion per element; bound by the exponential unit
+        const FoldedScale f = etq_folded_scale(rmax, m_s, K);
+        byte = f.byte;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            uint32_t word = 0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float lo = ex2_approx(__fmaf_rn(r[q * 8 + 2 * i], f.c1, f.c0e));
+                const float hi = ex2_approx(__fmaf_rn(r[q * 8 + 2 * i + 1], f.c1, f.c0e));
+                word |= (cvt_e2m1x2(lo, hi) & 0xffu) << (8 * i);
+            }
+            w[q] = f.live ? word : 0u;
         }
     } else {
         float p[32];

@@ -43,3 +43,4 @@ def test_host_side_validation_needs_no_gpu():
     assert L.efq_probgen(20, 64, 16, 4, 64, 1.0, ctypes.byref(p), 16, 16, None) == 3   # misaligned scores
     assert L.efq_probgen(16, 66, 16, 4, 64, 1.0, ctypes.byref(p), 16, 16, None) == 3   # ld % 4 != 0
     assert L.exp_then_quantize_probgen(16, 64, 16, 4, 64, 1.0, 5, 16, 16, None) == 1   # bad scale_mode
+    assert L.exp_then_quantize_probgen(16, 64, 16, 4, 64, 1.0, -1, 16, 16, None) == 1
