@@ -200,7 +200,9 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     const uint32_t tmem = sm->tmem_base;
     const bool run = sm->abort_flag == 0 && n_tiles > 0;
 
-    // register budget: the probability warpgroups take what the producer/issuer warpgroup gives up
+    // Register budget: the probability warpgroups take what the other two give up.  setmaxnreg moves registers
+    // inside the CTA's own allocation only (512 threads x 128 at launch = 16 x 128 per lane), so the budgets must
+    // add up to no more than that: 4 x 56 + 8 x 200 + 4 x 56 = 2048.  A role that asks for more waits for good.
     if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
     if (run && warp == 0 && lane == 0) {
