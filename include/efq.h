@@ -157,6 +157,27 @@ efq_status_t efq_attention_fwd_quantized(float* o, int B, int Hq, int Hkv, int64
                                          void* workspace, size_t workspace_bytes, const efq_debug_t* debug,
                                          void* stream);
 
+/* Packed variable-length batch (cross-attention, prefill of mixed lengths, decode steps; Sec. 4 names cross-attention
+ * among the places the method applies).  The n_seqs sequences lie one after the other along the token axis:
+ *   q [total_q, Hq, d], k and v [total_k, Hkv, d] bf16, o [total_q, Hq, d] fp32, all DEVICE, token-major;
+ *   cu_seqlens_q / cu_seqlens_k: HOST arrays of n_seqs + 1 non-decreasing prefix sums starting at 0; sequence i owns
+ *   query tokens [cu_q[i], cu_q[i+1]) and key tokens [cu_k[i], cu_k[i+1]).
+ * Every sequence is an attention problem of its own (Algorithm 2 over its own keys; with `causal`, query i of a
+ * sequence sees its keys <= i + len_k - len_q, the rule of efq_attention_fwd); the operands of a sequence are
+ * quantised by themselves, so the result of a sequence equals efq_attention_fwd on that sequence alone, bit for
+ * bit.  A sequence without queries is skipped; one without keys gets zero rows.  `producer` as for
+ * efq_attention_fwd_quantized.  The sequences are launched one after the other on `stream` (four kernels each)
+ * and share one workspace slot: efq_attention_varlen_workspace_bytes() gives the size (0 for invalid arguments).
+ * Asynchronous; efq_poll_status(workspace, stream) reports the first device-side problem of any sequence.
+ * Errors: INVALID_ARG (null pointer, n_seqs < 0, prefix sums not starting at 0 or decreasing, bad params),
+ * UNSUPPORTED (d != 128, a sequence too long for the 32-bit tile coordinates), ALIGNMENT, WORKSPACE, ARCH, CUDA. */
+size_t efq_attention_varlen_workspace_bytes(const int64_t* cu_seqlens_q, const int64_t* cu_seqlens_k, int n_seqs, int Hq,
+                                            int Hkv, int d);
+efq_status_t efq_attention_fwd_varlen(const void* q, const void* k, const void* v, float* o, const int64_t* cu_seqlens_q,
+                                      const int64_t* cu_seqlens_k, int n_seqs, int Hq, int Hkv, int d, int causal,
+                                      float softmax_scale, int producer, const efq_params_t* params, void* workspace,
+                                      size_t workspace_bytes, void* stream);
+
 /* End-to-end form with HOST inputs and output: copies q/k/v from (preferably pinned) host
  * memory into caller-owned device staging buffers, runs the forward selected by `producer`
  * (0 = EFQ, 1 = exp-then-quantize scale4, 2 = exp-then-quantize scale6), copies o back, all on

@@ -24,6 +24,7 @@ STATIC_SCRATCH_BYTES = 4 << 20
 EXPORTS = ["efq_probgen", "exp_then_quantize_probgen", "efq_attention_workspace_bytes", "efq_attention_fwd",
            "exp_then_quantize_attention_fwd", "efq_quantize_qkv", "efq_attention_fwd_quantized",
            "efq_attention_fwd_host", "efq_attention_fwd_host_pipelined", "efq_attention_fwd_static", "efq_poll_status",
+           "efq_attention_varlen_workspace_bytes", "efq_attention_fwd_varlen",
            "efq_exact_attention_fwd", "efq_relative_error", "efq_calibrate",
            "efq_fp4_mma_peak_probe", "efq_stage_microbench", "efq_attention_fwd_inject_timeout", "efq_status_string",
            "efq_version"]
@@ -81,6 +82,11 @@ def lib() -> C.CDLL:
         L.efq_attention_fwd_host_pipelined.restype = i32
         L.efq_attention_fwd_host_pipelined.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i64, i64, i32, i32,
                                                        f32, i32, C.POINTER(EfqParams), vp, C.c_size_t, i32, vp, vp, vp]
+        L.efq_attention_varlen_workspace_bytes.restype = C.c_size_t
+        L.efq_attention_varlen_workspace_bytes.argtypes = [C.POINTER(i64), C.POINTER(i64), i32, i32, i32, i32]
+        L.efq_attention_fwd_varlen.restype = i32
+        L.efq_attention_fwd_varlen.argtypes = [vp, vp, vp, vp, C.POINTER(i64), C.POINTER(i64), i32, i32, i32, i32, i32, f32,
+                                               i32, C.POINTER(EfqParams), vp, C.c_size_t, vp]
         L.efq_attention_fwd_static.restype = i32
         L.efq_attention_fwd_static.argtypes = [vp, vp, vp, vp, i32, i32, i32, i64, i64, i32, i32, f32,
                                                C.POINTER(EfqParams), vp]
@@ -259,6 +265,32 @@ def efq_attention_fwd_quantized(o, shape, workspace, causal: bool = False, softm
                                            workspace.data_ptr(), workspace.numel(),
                                            C.byref(debug.c) if debug is not None else None, _stream(stream))
     _check(st, "efq_attention_fwd_quantized")
+    return o
+
+
+def efq_attention_fwd_varlen(q, k, v, cu_seqlens_q, cu_seqlens_k, causal: bool = False, softmax_scale: float = 0.0,
+                             producer: int = 0, params=None, workspace=None, stream=None):
+    """Packed variable-length batch: q [total_q, Hq, d], k, v [total_k, Hkv, d] bf16 CUDA tensors (token-major);
+    cu_seqlens_*: sequences of n_seqs + 1 host integers.  Returns o [total_q, Hq, d] fp32."""
+    total_q, Hq, d = q.shape
+    total_k, Hkv, _ = k.shape
+    assert q.is_contiguous() and k.is_contiguous() and v.is_contiguous() and v.shape == k.shape
+    n = len(cu_seqlens_q) - 1
+    assert len(cu_seqlens_k) == n + 1 and int(cu_seqlens_q[-1]) == total_q and int(cu_seqlens_k[-1]) == total_k
+    cq = (C.c_int64 * (n + 1))(*[int(x) for x in cu_seqlens_q])
+    ck = (C.c_int64 * (n + 1))(*[int(x) for x in cu_seqlens_k])
+    if workspace is None:
+        nbytes = lib().efq_attention_varlen_workspace_bytes(cq, ck, n, Hq, Hkv, d)
+        if nbytes == 0:
+            raise EfqError(1, "efq_attention_varlen_workspace_bytes")
+        workspace = torch.empty(nbytes, dtype=torch.uint8, device=q.device)
+    o = torch.empty((total_q, Hq, d), dtype=torch.float32, device=q.device)
+    p = _params(params)
+    st = lib().efq_attention_fwd_varlen(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), cq, ck, n, Hq, Hkv, d,
+                                        int(bool(causal)), float(softmax_scale), int(producer),
+                                        C.byref(p) if p is not None else None, workspace.data_ptr(), workspace.numel(),
+                                        _stream(stream))
+    _check(st, "efq_attention_fwd_varlen")
     return o
 
 

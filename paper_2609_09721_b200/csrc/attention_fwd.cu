@@ -36,10 +36,10 @@
 
 namespace efq {
 
-cudaError_t launch_quantize_rows(const void* x, int64_t n_heads, int64_t S, int64_t S_pad, uint8_t* codes, uint8_t* sf,
-                                 cudaStream_t stream);
-cudaError_t launch_quantize_v(const void* v, int64_t n_heads, int64_t S, int64_t S_pad, uint8_t* vt_codes, uint8_t* sf,
-                              cudaStream_t stream);
+cudaError_t launch_quantize_rows(const void* x, int64_t n_heads, int64_t S, int64_t S_pad, int64_t head_stride,
+                                 int64_t row_stride, uint8_t* codes, uint8_t* sf, cudaStream_t stream);
+cudaError_t launch_quantize_v(const void* v, int64_t n_heads, int64_t S, int64_t S_pad, int64_t head_stride,
+                              int64_t row_stride, uint8_t* vt_codes, uint8_t* sf, cudaStream_t stream);
 
 namespace {
 
@@ -95,6 +95,7 @@ struct FwdParams {
     const uint8_t* sf_k;      // [B*Hkv*Sk_pad/128][512]
     const uint8_t* sf_v;
     float* o;
+    int64_t o_head, o_row;    // strides of o in elements: row i of (batch b, head h) starts at o[(b * Hq + h) * o_head + i * o_row]
     uint32_t* status;
     efq_debug_t dbg;
     int has_dbg;
@@ -482,7 +483,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             if (grow < P.Sq) {
                 const float l = __uint_as_float(lcol);
                 const float inv = l > 0.0f ? 1.0f / l : 0.0f;
-                float4* dst = reinterpret_cast<float4*>(P.o + ((bh * P.Sq + grow) * 128 + 64 * group));
+                float4* dst = reinterpret_cast<float4*>(P.o + (bh * P.o_head + grow * P.o_row + 64 * group));
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
                     float4 v;
@@ -497,7 +498,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     } else if (sm->abort_flag == 0) {
         // no visible key for the whole tile: rows are zero
         if (grow < P.Sq) {
-            float4* dst = reinterpret_cast<float4*>(P.o + ((bh * P.Sq + grow) * 128 + 64 * group));
+            float4* dst = reinterpret_cast<float4*>(P.o + (bh * P.o_head + grow * P.o_row + 64 * group));
             for (int i = 0; i < 16; ++i) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
     }
@@ -603,10 +604,14 @@ cudaError_t launch_main(bool debug, bool fix8, dim3 grid, size_t smem, cudaStrea
 efq_status_t attention_impl(const void* q, const void* k, const void* v, float* o, int B, int Hq, int Hkv, int64_t Sq,
                             int64_t Sk, int d, int causal, float softmax_scale, int producer, float tau, float h,
                             void* workspace, size_t workspace_bytes, const efq_debug_t* debug, cudaStream_t stream,
-                            bool do_quantize, bool do_forward, bool inject_skip_loads = false, float rescale_threshold = 0.0f)
+                            bool do_quantize, bool do_forward, bool inject_skip_loads = false, float rescale_threshold = 0.0f,
+                            bool token_major = false)
 {
+    // token_major: q, k, v are [S, H, d] and o is [Sq, Hq, d] (one sequence of a packed batch; B must be 1);
+    // otherwise [B, H, S, d]
     if (!q || !k || !v || !o) return EFQ_ERR_INVALID_ARG;
     if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0 || Hq % Hkv != 0) return EFQ_ERR_INVALID_ARG;
+    if (token_major && B != 1) return EFQ_ERR_INVALID_ARG;
     if (d != 128) return EFQ_ERR_UNSUPPORTED;
     if (!shape_ok(B, Hq, Hkv, Sq, Sk, d)) return EFQ_ERR_UNSUPPORTED;
     if (!(softmax_scale > 0.0f)) softmax_scale = static_cast<float>(1.0 / sqrt(static_cast<double>(d)));
@@ -625,9 +630,11 @@ efq_status_t attention_impl(const void* q, const void* k, const void* v, float* 
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     if (do_quantize) {
         if (cudaMemsetAsync(ws + w.status, 0, 1024, stream) != cudaSuccess) return EFQ_ERR_CUDA;
-        if (launch_quantize_rows(q, static_cast<int64_t>(B) * Hq, Sq, w.Sq_pad, ws + w.qc, ws + w.qsf, stream) != cudaSuccess) return EFQ_ERR_CUDA;
-        if (launch_quantize_rows(k, static_cast<int64_t>(B) * Hkv, Sk, w.Sk_pad, ws + w.kc, ws + w.ksf, stream) != cudaSuccess) return EFQ_ERR_CUDA;
-        if (launch_quantize_v(v, static_cast<int64_t>(B) * Hkv, Sk, w.Sk_pad, ws + w.vt, ws + w.vsf, stream) != cudaSuccess) return EFQ_ERR_CUDA;
+        const int64_t qh = token_major ? 128 : Sq * 128, qr = token_major ? static_cast<int64_t>(Hq) * 128 : 128;
+        const int64_t kh = token_major ? 128 : Sk * 128, kr = token_major ? static_cast<int64_t>(Hkv) * 128 : 128;
+        if (launch_quantize_rows(q, static_cast<int64_t>(B) * Hq, Sq, w.Sq_pad, qh, qr, ws + w.qc, ws + w.qsf, stream) != cudaSuccess) return EFQ_ERR_CUDA;
+        if (launch_quantize_rows(k, static_cast<int64_t>(B) * Hkv, Sk, w.Sk_pad, kh, kr, ws + w.kc, ws + w.ksf, stream) != cudaSuccess) return EFQ_ERR_CUDA;
+        if (launch_quantize_v(v, static_cast<int64_t>(B) * Hkv, Sk, w.Sk_pad, kh, kr, ws + w.vt, ws + w.vsf, stream) != cudaSuccess) return EFQ_ERR_CUDA;
     }
     if (!do_forward) return EFQ_OK;
 
@@ -642,6 +649,8 @@ efq_status_t attention_impl(const void* q, const void* k, const void* v, float* 
     P.K = producer == 3 ? make_producer_consts_lut(softmax_scale) : make_producer_consts(softmax_scale, tau, h);
     P.sf_q = ws + w.qsf; P.sf_k = ws + w.ksf; P.sf_v = ws + w.vsf;
     P.o = o;
+    P.o_head = token_major ? 128 : Sq * 128;
+    P.o_row = token_major ? static_cast<int64_t>(Hq) * 128 : 128;
     P.status = reinterpret_cast<uint32_t*>(ws + w.status);
     P.inject_skip_loads = inject_skip_loads ? 1 : 0;
     P.rescale_threshold = rescale_threshold;
@@ -874,6 +883,85 @@ extern "C" efq_status_t efq_attention_fwd_host_pipelined(const void* q_host, con
     if (cudaEventRecord(ev, s_out) != cudaSuccess || cudaStreamWaitEvent(s_c, ev, 0) != cudaSuccess) return fail(EFQ_ERR_CUDA);
     cudaEventDestroy(ev);
     return EFQ_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Packed variable-length batch: the sequences of the batch lie one after the other along the token axis
+// ------------------------------------------------------------------------------------------------
+namespace efq {
+namespace {
+// checks the two prefix arrays and returns the workspace slot of the largest sequence (0: nothing to do; -1: bad input)
+int64_t varlen_slot_bytes(const int64_t* cu_q, const int64_t* cu_k, int n_seqs, int Hq, int Hkv, int d, efq_status_t& st)
+{
+    st = EFQ_OK;
+    if (!cu_q || !cu_k || n_seqs < 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0) { st = EFQ_ERR_INVALID_ARG; return -1; }
+    if (d != 128) { st = EFQ_ERR_UNSUPPORTED; return -1; }
+    if (n_seqs > 0 && (cu_q[0] != 0 || cu_k[0] != 0)) { st = EFQ_ERR_INVALID_ARG; return -1; }
+    size_t slot = 0;
+    for (int s = 0; s < n_seqs; ++s) {
+        const int64_t lq = cu_q[s + 1] - cu_q[s], lk = cu_k[s + 1] - cu_k[s];
+        if (lq < 0 || lk < 0) { st = EFQ_ERR_INVALID_ARG; return -1; }
+        if (lq == 0 || lk == 0) continue;
+        if (!shape_ok(1, Hq, Hkv, lq, lk, d)) { st = EFQ_ERR_UNSUPPORTED; return -1; }
+        const size_t need = plan_workspace(1, Hq, Hkv, lq, lk).total;
+        if (need > slot) slot = need;
+    }
+    return static_cast<int64_t>(slot);
+}
+}  // namespace
+}  // namespace efq
+
+extern "C" size_t efq_attention_varlen_workspace_bytes(const int64_t* cu_seqlens_q, const int64_t* cu_seqlens_k, int n_seqs,
+                                                       int Hq, int Hkv, int d)
+{
+    efq_status_t st;
+    const int64_t slot = efq::varlen_slot_bytes(cu_seqlens_q, cu_seqlens_k, n_seqs, Hq, Hkv, d, st);
+    return slot < 0 ? 0 : static_cast<size_t>(slot) + 1024;
+}
+
+extern "C" efq_status_t efq_attention_fwd_varlen(const void* q, const void* k, const void* v, float* o,
+                                                 const int64_t* cu_seqlens_q, const int64_t* cu_seqlens_k, int n_seqs,
+                                                 int Hq, int Hkv, int d, int causal, float softmax_scale, int producer,
+                                                 const efq_params_t* params, void* workspace, size_t workspace_bytes,
+                                                 void* stream)
+{
+    float tau, h, threshold;
+    bool lut;
+    efq_status_t st;
+    if (!read_params(params, tau, h, lut, threshold, st)) return st;
+    if (producer == 0 && lut) producer = 3;
+    if (producer < 0 || producer > 4) return EFQ_ERR_INVALID_ARG;
+    const int64_t slot = efq::varlen_slot_bytes(cu_seqlens_q, cu_seqlens_k, n_seqs, Hq, Hkv, d, st);
+    if (slot < 0) return st;
+    if (n_seqs == 0 || cu_seqlens_q[n_seqs] == 0) return EFQ_OK;     // no query token: nothing to write
+    if (!q || !k || !v || !o) return EFQ_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes < static_cast<size_t>(slot) + 1024) return EFQ_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    uint32_t* agg = reinterpret_cast<uint32_t*>(ws + slot);          // first problem seen by any sequence
+    if (cudaMemsetAsync(agg, 0, 4, s) != cudaSuccess) return EFQ_ERR_CUDA;
+    if (cudaMemsetAsync(ws, 0, 4, s) != cudaSuccess) return EFQ_ERR_CUDA;
+    for (int i = 0; i < n_seqs; ++i) {
+        const int64_t q0 = cu_seqlens_q[i], k0 = cu_seqlens_k[i];
+        const int64_t lq = cu_seqlens_q[i + 1] - q0, lk = cu_seqlens_k[i + 1] - k0;
+        if (lq == 0) continue;
+        float* oi = o + q0 * Hq * 128;
+        if (lk == 0) {               // no key at all: the rows are zero, as for a causal row that sees nothing
+            if (cudaMemsetAsync(oi, 0, static_cast<size_t>(lq) * Hq * 128 * sizeof(float), s) != cudaSuccess) return EFQ_ERR_CUDA;
+            continue;
+        }
+        const uint16_t* qi = static_cast<const uint16_t*>(q) + q0 * Hq * 128;
+        const uint16_t* ki = static_cast<const uint16_t*>(k) + k0 * Hkv * 128;
+        const uint16_t* vi = static_cast<const uint16_t*>(v) + k0 * Hkv * 128;
+        // the sequences run in stream order, so one workspace slot serves them all
+        st = efq::attention_impl(qi, ki, vi, oi, 1, Hq, Hkv, lq, lk, d, causal, softmax_scale, producer, tau, h, ws,
+                                 static_cast<size_t>(slot), nullptr, s, true, true, false, threshold, true);
+        if (st != EFQ_OK) return st;
+        efq::merge_status_kernel<<<1, 1, 0, s>>>(agg, reinterpret_cast<const uint32_t*>(ws), 0);
+        if (cudaGetLastError() != cudaSuccess) return EFQ_ERR_CUDA;
+    }
+    efq::merge_status_kernel<<<1, 1, 0, s>>>(reinterpret_cast<uint32_t*>(ws), agg, 1);
+    return cudaGetLastError() == cudaSuccess ? EFQ_OK : EFQ_ERR_CUDA;
 }
 
 extern "C" efq_status_t efq_poll_status(void* workspace, void* stream)

@@ -56,10 +56,11 @@ __device__ __forceinline__ void mxfp4_block(const uint32_t (&w)[16], uint4& code
 
 __device__ __forceinline__ uint32_t sf_tile_offset(uint32_t r, uint32_t b) { return (r & 31u) * 16u + (r >> 5) * 4u + b; }
 
-// One thread per (row, 32-wide block along d); d = 128.
+// One thread per (row, 32-wide block along d); d = 128.  The input is addressed by strides in elements:
+// element (head, row, c) at x[head * head_stride + row * row_stride + c].
 __global__ void __launch_bounds__(256)
 quantize_rows_kernel(const __nv_bfloat16* __restrict__ x, int64_t n_heads, int64_t S, int64_t S_pad,
-                     uint8_t* __restrict__ codes, uint8_t* __restrict__ sf)
+                     int64_t head_stride, int64_t row_stride, uint8_t* __restrict__ codes, uint8_t* __restrict__ sf)
 {
     const int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     const int64_t total = n_heads * S_pad * 4;
@@ -71,7 +72,7 @@ quantize_rows_kernel(const __nv_bfloat16* __restrict__ x, int64_t n_heads, int64
     uint4 c = make_uint4(0, 0, 0, 0);
     uint32_t byte = 0;
     if (row < S) {
-        const uint4* src = reinterpret_cast<const uint4*>(x + (head * S + row) * 128 + blk * 32);
+        const uint4* src = reinterpret_cast<const uint4*>(x + head * head_stride + row * row_stride + blk * 32);
         uint32_t w[16];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -88,20 +89,20 @@ quantize_rows_kernel(const __nv_bfloat16* __restrict__ x, int64_t n_heads, int64
 // One thread per (32-key block, channel); consecutive threads take consecutive channels.
 __global__ void __launch_bounds__(128)
 quantize_v_kernel(const __nv_bfloat16* __restrict__ v, int64_t n_heads, int64_t S, int64_t S_pad,
-                  uint8_t* __restrict__ vt_codes, uint8_t* __restrict__ sf)
+                  int64_t head_stride, int64_t row_stride, uint8_t* __restrict__ vt_codes, uint8_t* __restrict__ sf)
 {
     const int ch = threadIdx.x;                               // 0..127
     const int64_t kb = blockIdx.x;                            // key block over all heads
     const int64_t blocks_per_head = S_pad / 32;
     const int64_t head = kb / blocks_per_head;
     const int64_t kblk = kb - head * blocks_per_head;
-    const uint16_t* src = reinterpret_cast<const uint16_t*>(v) + (head * S + kblk * 32) * 128 + ch;
+    const uint16_t* src = reinterpret_cast<const uint16_t*>(v) + head * head_stride + kblk * 32 * row_stride + ch;
     uint32_t w[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
         const int64_t k0 = kblk * 32 + 2 * i;
-        uint32_t lo = k0 < S ? __ldg(src + (2 * i) * 128) : 0u;
-        uint32_t hi = k0 + 1 < S ? __ldg(src + (2 * i + 1) * 128) : 0u;
+        uint32_t lo = k0 < S ? __ldg(src + (2 * i) * row_stride) : 0u;
+        uint32_t hi = k0 + 1 < S ? __ldg(src + (2 * i + 1) * row_stride) : 0u;
         w[i] = lo | (hi << 16);
     }
     uint4 c;
@@ -112,23 +113,23 @@ quantize_v_kernel(const __nv_bfloat16* __restrict__ v, int64_t n_heads, int64_t 
     sf[tile * 512 + sf_tile_offset(static_cast<uint32_t>(ch), static_cast<uint32_t>(kblk & 3))] = static_cast<uint8_t>(byte);
 }
 
-cudaError_t launch_quantize_rows(const void* x, int64_t n_heads, int64_t S, int64_t S_pad, uint8_t* codes, uint8_t* sf,
-                                 cudaStream_t stream)
+cudaError_t launch_quantize_rows(const void* x, int64_t n_heads, int64_t S, int64_t S_pad, int64_t head_stride,
+                                 int64_t row_stride, uint8_t* codes, uint8_t* sf, cudaStream_t stream)
 {
     const int64_t total = n_heads * S_pad * 4;
     if (total == 0) return cudaSuccess;
     quantize_rows_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, stream>>>(
-        static_cast<const __nv_bfloat16*>(x), n_heads, S, S_pad, codes, sf);
+        static_cast<const __nv_bfloat16*>(x), n_heads, S, S_pad, head_stride, row_stride, codes, sf);
     return cudaGetLastError();
 }
 
-cudaError_t launch_quantize_v(const void* v, int64_t n_heads, int64_t S, int64_t S_pad, uint8_t* vt_codes, uint8_t* sf,
-                              cudaStream_t stream)
+cudaError_t launch_quantize_v(const void* v, int64_t n_heads, int64_t S, int64_t S_pad, int64_t head_stride,
+                              int64_t row_stride, uint8_t* vt_codes, uint8_t* sf, cudaStream_t stream)
 {
     const int64_t blocks = n_heads * (S_pad / 32);
     if (blocks == 0) return cudaSuccess;
     quantize_v_kernel<<<static_cast<unsigned>(blocks), 128, 0, stream>>>(static_cast<const __nv_bfloat16*>(v), n_heads, S,
-                                                                         S_pad, vt_codes, sf);
+                                                                         S_pad, head_stride, row_stride, vt_codes, sf);
     return cudaGetLastError();
 }
 

@@ -111,7 +111,8 @@ def test_small_shapes_efq(oracle, S, Hq, Hkv, causal, recipe):
     _check_dump(oracle, case, dump, _all_rows(case, head, 0, S), MEAN)
 
 
-@pytest.mark.parametrize("Sq,Sk,causal", [(128, 512, True), (100, 700, False), (260, 200, True), (64, 4096 + 88, True)])
+@pytest.mark.parametrize("Sq,Sk,causal", [(128, 512, True), (100, 700, False), (260, 200, True), (64, 4096 + 88, True),
+                                          (1, 4096 + 88, True), (1, 300, False), (3, 129, True)])   # the last three: decode steps
 def test_cross_shapes_sq_ne_sk(oracle, Sq, Sk, causal):
     case = inputs.AttentionCase("x", 1, 2, 1, Sq, Sk, 128, causal, 77, "iid")
     (q, k, v), (dq, dk, dv) = _case_tensors(case)
@@ -198,6 +199,63 @@ def test_exp_then_quantize_path(oracle, mode, path):
     _check_dump(oracle, case, dump, _all_rows(case, 1, 0, 640), MEAN, producer=path)
     exact = oracle.attention_rows(q, k, v, rows, True, case.softmax_scale, "exact")
     print(path, "rel-Frobenius vs exact =", np.linalg.norm(got - exact) / np.linalg.norm(exact))
+
+
+@pytest.mark.parametrize("causal,producer,params", [(True, 0, None), (False, 0, None), (True, 0, (0.0, 1.0, 1)), (True, 1, None)])
+def test_varlen_packed_batch(oracle, causal, producer, params):
+    """Sequences of mixed lengths packed along the token axis: each equals the forward of that sequence alone."""
+    Hq, Hkv = 4, 2
+    lens = [(300, 300), (1, 700), (128, 128), (0, 50), (77, 1000), (40, 0), (200, 64)]
+    qs, ks, vs, alone = [], [], [], []
+    for n, (lq, lk) in enumerate(lens):
+        case = inputs.AttentionCase("v", 1, Hq, Hkv, max(lq, 1), max(lk, 1), 128, causal, 300 + n, "k_outliers")
+        (q, k, v), (dq, dk, dv) = _case_tensors(case)
+        qs.append(dq[0, :, :lq].permute(1, 0, 2))        # [len, H, d]
+        ks.append(dk[0, :, :lk].permute(1, 0, 2))
+        vs.append(dv[0, :, :lk].permute(1, 0, 2))
+        alone.append((case, (q, k, v), (dq, dk, dv)))
+    qp, kp, vp = (torch.cat(t, 0).contiguous() for t in (qs, ks, vs))
+    cu_q = np.concatenate([[0], np.cumsum([a for a, _ in lens])])
+    cu_k = np.concatenate([[0], np.cumsum([b for _, b in lens])])
+    nbytes = binding.lib().efq_attention_varlen_workspace_bytes(
+        (binding.C.c_int64 * len(cu_q))(*cu_q.tolist()), (binding.C.c_int64 * len(cu_k))(*cu_k.tolist()), len(lens), Hq, Hkv, 128)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    o = binding.efq_attention_fwd_varlen(qp, kp, vp, cu_q, cu_k, causal, 0.0, producer, params, workspace=ws)
+    assert binding.efq_poll_status(ws) == 0
+    path = {(0, None): "efq", (0, (0.0, 1.0, 1)): "efq_lut", (1, None): "etq"}[(producer, params)]
+    for n, (lq, lk) in enumerate(lens):
+        got = o[cu_q[n]:cu_q[n + 1]]                     # [lq, Hq, d]
+        if lq == 0:
+            continue
+        if lk == 0:
+            assert torch.all(got == 0)
+            continue
+        case, (q, k, v), (dq, dk, dv) = alone[n]
+        if producer == 0:
+            one = binding.efq_attention_fwd(dq, dk, dv, causal, 0.0, params)
+        else:
+            one = binding.exp_then_quantize_attention_fwd(dq, dk, dv, causal, 0.0, 0)
+        assert torch.equal(got.permute(1, 0, 2), one[0]), f"sequence {n} differs from the forward of that sequence alone"
+        rows = np.array([(0, h, i) for h in range(Hq) for i in range(lq)], np.int64)
+        want = oracle.attention_rows(q, k, v, rows, causal, case.softmax_scale, path)
+        err = np.abs(got.permute(1, 0, 2).reshape(-1, 128).cpu().numpy() - want).max()
+        assert err <= (TOL_O if producer == 0 else 5e-3)
+
+
+def test_varlen_argument_errors():
+    q = torch.zeros((8, 2, 128), dtype=torch.bfloat16, device="cuda")
+    good = [0, 8]
+    with pytest.raises(binding.EfqError) as e:
+        binding.efq_attention_fwd_varlen(q, q, q, [1, 8], good)           # prefix sums must start at 0
+    assert e.value.status == 1
+    with pytest.raises(binding.EfqError) as e:
+        binding.efq_attention_fwd_varlen(q, q, q, [0, 9, 8], [0, 4, 8])   # decreasing
+    assert e.value.status == 1
+    with pytest.raises(binding.EfqError) as e:
+        binding.efq_attention_fwd_varlen(q, q, q, good, good, workspace=torch.empty(1024, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 4
+    o = binding.efq_attention_fwd_varlen(q[:0], q[:0], q[:0], [0], [0])   # empty batch: nothing to do
+    assert o.shape == (0, 2, 128)
 
 
 def _sampled_parity(oracle, case, n_random, label):
