@@ -294,7 +294,7 @@ def run_cuda(args):
 
     # timed variants: the library's producer id (0 EFQ, 1 exp-then-quantize, 4 the same with the scale folded into ex2)
     # and the efq_params_t that goes with it
-    VARIANTS = {"efq": (0, None), "etq": (1, None), "etq_folded": (4, None), "efq_lut": (0, LUT), "efq_lazy": (0, LAZY)}
+    VARIANTS = {"efq": (0, None), "etq": (1, None), "etq_folded": (4, None), "etq_hybrid": (5, None), "efq_lut": (0, LUT), "efq_lazy": (0, LAZY)}
 
     def step(variant="efq", ev=None):
         producer, prm = VARIANTS[variant]
@@ -341,6 +341,7 @@ def run_cuda(args):
         raise SystemExit(f"bench.py: device status {status} after the timed region")
     etq_ms_step, etq_ms_main, _ = timed("etq", max(3, args.steps // 2), 3)
     etqf_ms_step, etqf_ms_main, _ = timed("etq_folded", max(3, args.steps // 2), 3)
+    etqh_ms_step, etqh_ms_main, _ = timed("etq_hybrid", max(3, args.steps // 2), 3)
     lut_ms_step, lut_ms_main, _ = timed("efq_lut", max(3, args.steps // 4), 3)
     lazy_ms_step, lazy_ms_main, _ = timed("efq_lazy", max(3, args.steps // 4), 3)
 
@@ -409,10 +410,11 @@ def run_cuda(args):
         t_efq = stage_time(lambda: binding.efq_probgen(sc, rm, 1.0, None, codes, scl))
         t_etq = stage_time(lambda: binding.exp_then_quantize_probgen(sc, rm, 1.0, 0, codes, scl))
         t_etqf = stage_time(lambda: binding.exp_then_quantize_probgen(sc, rm, 1.0, 2, codes, scl))
+        t_etqh = stage_time(lambda: binding.exp_then_quantize_probgen(sc, rm, 1.0, 3, codes, scl))
         t_lut = stage_time(lambda: binding.efq_probgen(sc, rm, 1.0, LUT, codes, scl))
         stage = {"workload": "probgen 4096x16384 fp32 (device-generated N(0,9), timing only)", "bytes_per_launch": nbytes,
                  "efq_ms": t_efq, "efq_gbs": nbytes / t_efq / 1e6, "etq_ms": t_etq, "etq_gbs": nbytes / t_etq / 1e6,
-                 "etq_folded_ms": t_etqf, "etq_folded_gbs": nbytes / t_etqf / 1e6, "efq_lut_ms": t_lut, "efq_lut_gbs": nbytes / t_lut / 1e6}
+                 "etq_folded_ms": t_etqf, "etq_folded_gbs": nbytes / t_etqf / 1e6, "etq_hybrid_ms": t_etqh, "etq_hybrid_gbs": nbytes / t_etqh / 1e6, "efq_lut_ms": t_lut, "efq_lut_gbs": nbytes / t_lut / 1e6}
 
     # accuracy beside the speed: relative Frobenius error of each producer's output against FP32 attention on
     # the unquantised inputs, on the whole benchmarked problem (reference kernel: plain CUDA cores, run once)
@@ -426,7 +428,7 @@ def run_cuda(args):
                     "reference_kernel_s": t_ref}
         binding.efq_quantize_qkv(dq, dk, dv, ws)
         for name, prod, prm in (("efq", 0, None), ("exp_then_quantize", 1, None), ("exp_then_quantize_scale6", 2, None),
-                                ("exp_then_quantize_folded", 4, None),
+                                ("exp_then_quantize_folded", 4, None), ("exp_then_quantize_hybrid", 5, None),
                                 ("efq_lut", 0, LUT), ("efq_mmlu", 0, (-2.90, 2.00)), ("efq_balance", 0, (-2.10, 2.70)),
                                 ("efq_thresholded_rescale_T4", 0, LAZY)):
             binding.efq_attention_fwd_quantized(o, shape, ws, case.causal, 0.0, prod, prm)
@@ -450,7 +452,7 @@ def run_cuda(args):
         peak_ms = a.elapsed_time(b)
         ok = bool((sink.cpu().numpy().view(np.uint32) != 0xdeadbeef).all())
         per_clk = {}
-        for name, prod in (("efq", 0), ("etq", 1), ("etq_folded", 4), ("efq_lut", 3)):
+        for name, prod in (("efq", 0), ("etq", 1), ("etq_folded", 4), ("etq_hybrid", 5), ("efq_lut", 3)):
             binding.efq_stage_microbench(prod, 2 * sms, 200)
             cyc = binding.efq_stage_microbench(prod, 2 * sms, 2000)
             torch.cuda.synchronize()
@@ -506,6 +508,10 @@ def run_cuda(args):
                                      "main_kernel_ms": etqf_ms_main, "efq_speedup": etqf_ms_step / ms_step,
                                      "note": "scale_mode 2: block scale folded into the exponential (one FMA + one ex2 per "
                                              "score, no FP32 probability); the strongest exponential baseline in this build"},
+        "exp_then_quantize_hybrid": {"value": flops / (etqh_ms_step * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": etqh_ms_step,
+                                     "main_kernel_ms": etqh_ms_main, "efq_speedup": etqh_ms_step / ms_step,
+                                     "note": "scale_mode 3: scale_mode 2 with 2 of 8 exponentials by a cubic polynomial on the "
+                                             "FMA pipe (takes load off MUFU; does not pay in the fused kernel)"},
         "efq_lut": {"value": flops / (lut_ms_step * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": lut_ms_step,
                     "main_kernel_ms": lut_ms_main, "note": "variant 1: 16-level index + folding table (accuracy ablation)"},
         "efq_thresholded_rescale": {"value": flops / (lazy_ms_step * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": lazy_ms_step,

@@ -109,7 +109,12 @@ efq_status_t efq_probgen(const float* scores, int64_t ld, const float* row_max, 
  * scale_mode 2 is scale_mode 0 in its fastest form on this machine: the same mathematics with the scale folded
  * into the exponential, p 2^-e = 2^(x log2(e) - e), so that no FP32 probability is formed either - one FMA, one
  * ex2 and half a conversion per element, bound by the exponential unit (16 per clock per SM).  Results agree
- * with scale_mode 0 except at rounding knife-edges. */
+ * with scale_mode 0 except at rounding knife-edges.
+ * scale_mode 3 is scale_mode 2 with 2 of every 8 exponentials computed on the FMA pipe (floor, cubic polynomial
+ * of the fraction with relative error 8.6e-5, exponent insertion) to take load off the exponential unit.  Measured
+ * on B200 it gains 3 % in the register-resident stage and loses 6 % in the fused forward, where issue slots and
+ * not the exponential unit are short; it is kept as the record of that comparison.  Codes differ from
+ * scale_mode 0 on a few elements in ten thousand (the polynomial's error against the E2M1 rounding step). */
 efq_status_t exp_then_quantize_probgen(const float* scores, int64_t ld, const float* row_max, int64_t rows,
                                        int64_t cols, float score_scale, int scale_mode, uint8_t* codes,
                                        uint8_t* scales, void* stream);
@@ -148,7 +153,7 @@ efq_status_t exp_then_quantize_attention_fwd(const void* q, const void* k, const
  * efq_quantize_qkv: operand preparation only (bf16 -> MXFP4 into the workspace; resets the status word).
  * efq_attention_fwd_quantized: the fused forward on a workspace prepared by efq_quantize_qkv for the
  * same shape; producer 0 = EFQ (with params->variant 1: EFQ-LUT), 1 = exp-then-quantize scale4, 2 = exp-then-quantize
- * scale6, 4 = exp-then-quantize scale4 with the scale folded into the exponential (scale_mode 2).
+ * scale6, 4 = exp-then-quantize scale4 with the scale folded into the exponential (scale_mode 2), 5 = scale_mode 3.
  * Arguments, layouts and errors as for efq_attention_fwd. */
 efq_status_t efq_quantize_qkv(const void* q, const void* k, const void* v, int B, int Hq, int Hkv, int64_t Sq,
                               int64_t Sk, int d, void* workspace, size_t workspace_bytes, void* stream);
@@ -278,7 +283,7 @@ efq_status_t efq_fp4_mma_peak_probe(uint32_t* sink, int num_ctas, int iters, dou
 
 /* In-SM microbenchmark of the probability producers (Algorithm 1 versus exp-then-quantize) on register-resident
  * scores: 256 threads per CTA, each coding one 32-key block per iteration, no memory traffic.
- *   producer 0 = EFQ (params or EFQ-Mean), 1 = exp-then-quantize scale4, 2 = scale6, 3 = EFQ-LUT, 4 = scale4 folded
+ *   producer 0 = EFQ (params or EFQ-Mean), 1 = exp-then-quantize scale4, 2 = scale6, 3 = EFQ-LUT, 4 = scale4 folded, 5 = scale4 folded + polynomial
  *   sink    u32 [num_ctas * 256], device (keeps the work alive)
  *   cycles  i64 [num_ctas], device: clock cycles CTA c spent on its `iters` iterations
  * Elements per clock per SM = resident CTAs per SM * 256 * 32 * iters / cycles. */

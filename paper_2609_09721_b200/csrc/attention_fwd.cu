@@ -670,6 +670,7 @@ efq_status_t attention_impl(const void* q, const void* k, const void* v, float* 
         case 2: e = launch_main<2>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
         case 3: e = launch_main<3>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
         case 4: e = launch_main<4>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
+        case 5: e = launch_main<5>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
         default: return EFQ_ERR_INVALID_ARG;
     }
     return e == cudaSuccess ? EFQ_OK : EFQ_ERR_CUDA;
@@ -685,7 +686,7 @@ extern "C" size_t efq_attention_workspace_bytes(int B, int Hq, int Hkv, int64_t 
 }
 
 // Producer ids inside the library: 0 = EFQ (affine rule), 1 / 2 = exp-then-quantize scale4 / scale6, 3 = EFQ-LUT,
-// 4 = exp-then-quantize scale4 with the scale folded into the exponential.
+// 4 = exp-then-quantize scale4 with the scale folded into the exponential, 5 = the same with 2 of 8 exponentials by polynomial.
 static bool read_params(const efq_params_t* params, float& tau, float& h, bool& lut, float& threshold, efq_status_t& st)
 {
     tau = -3.06f;
@@ -725,8 +726,8 @@ extern "C" efq_status_t exp_then_quantize_attention_fwd(const void* q, const voi
                                                         float softmax_scale, int scale_mode, void* workspace,
                                                         size_t workspace_bytes, const efq_debug_t* debug, void* stream)
 {
-    if (scale_mode < 0 || scale_mode > 2) return EFQ_ERR_INVALID_ARG;
-    return efq::attention_impl(q, k, v, o, B, Hq, Hkv, Sq, Sk, d, causal, softmax_scale, scale_mode == 2 ? 4 : 1 + scale_mode, 0.0f, 1.0f,
+    if (scale_mode < 0 || scale_mode > 3) return EFQ_ERR_INVALID_ARG;
+    return efq::attention_impl(q, k, v, o, B, Hq, Hkv, Sq, Sk, d, causal, softmax_scale, scale_mode >= 2 ? scale_mode + 2 : 1 + scale_mode, 0.0f, 1.0f,
                                workspace, workspace_bytes, debug, static_cast<cudaStream_t>(stream), true, true);
 }
 
@@ -930,7 +931,7 @@ extern "C" efq_status_t efq_attention_fwd_varlen(const void* q, const void* k, c
     efq_status_t st;
     if (!read_params(params, tau, h, lut, threshold, st)) return st;
     if (producer == 0 && lut) producer = 3;
-    if (producer < 0 || producer > 4) return EFQ_ERR_INVALID_ARG;
+    if (producer < 0 || producer > 5) return EFQ_ERR_INVALID_ARG;
     const int64_t slot = efq::varlen_slot_bytes(cu_seqlens_q, cu_seqlens_k, n_seqs, Hq, Hkv, d, st);
     if (slot < 0) return st;
     if (n_seqs == 0 || cu_seqlens_q[n_seqs] == 0) return EFQ_OK;     // no query token: nothing to write

@@ -38,7 +38,8 @@ __device__ __forceinline__ float block_max32(const float* r)
 
 // 32 scores of one microscaling block -> 16 bytes of codes + scale byte.
 // PRODUCER: 0 = EFQ (affine rule), 1 / 2 = exp-then-quantize with the block maximum in [4, 8) / (3, 6],
-// 3 = EFQ-LUT, 4 = exp-then-quantize [4, 8) with the scale folded into the exponential.
+// 3 = EFQ-LUT, 4 = exp-then-quantize [4, 8) with the scale folded into the exponential, 5 = the same with 2 of 8
+// exponentials computed by a polynomial on the FMA pipe.
 //
 // EFQ (Algorithm 1), three FMA-pipe instructions per element, bit-identical to
 // c = floor(min(max(fma(r, A, Bb), 0), 7)):
@@ -88,20 +89,22 @@ __device__ __forceinline__ void produce32(const float* r, float rmax, float m_s,
             for (int i = 0; i < 8; ++i) word |= lut_code(r[q * 8 + i], A16, B16) << (4 * i);
             w[q] = word;
         }
-    } else if (PRODUCER == 4) {
+    } else if (PRODUCER == 4 || PRODUCER == 5) {
         // exp-then-quantize (block maximum in [4, 8)) with the scale folded into the exponential: one FMA, one ex2
-        // and half a conversion per element; bound by the exponential unit
+        // and half a conversion per element; bound by the exponential unit.  PRODUCER 5 moves 2 of every 8
+        // exponentials onto the FMA pipe (cubic polynomial).
         const FoldedScale f = etq_folded_scale(rmax, m_s, K);
         byte = f.byte;
+        auto ex2 = [&](const int i) {
+            const float t = __fmaf_rn(r[i], f.c1, f.c0e);
+            return (PRODUCER == 5 && ex2_by_poly(i)) ? ex2_poly3(t) : ex2_approx(t);
+        };
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             uint32_t word = 0;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float lo = ex2_approx(__fmaf_rn(r[q * 8 + 2 * i], f.c1, f.c0e));
-                const float hi = ex2_approx(__fmaf_rn(r[q * 8 + 2 * i + 1], f.c1, f.c0e));
-                word |= (cvt_e2m1x2(lo, hi) & 0xffu) << (8 * i);
-            }
+            for (int i = 0; i < 4; ++i)
+                word |= (cvt_e2m1x2(ex2(q * 8 + 2 * i), ex2(q * 8 + 2 * i + 1)) & 0xffu) << (8 * i);
             w[q] = f.live ? word : 0u;
         }
     } else {

@@ -135,6 +135,7 @@ extern "C" efq_status_t efq_stage_microbench(int producer, const efq_params_t* p
             break;
         case 1: efq::stage_kernel<1, false><<<num_ctas, 256, 0, s>>>(K, iters, sink, cycles); break;
         case 2: efq::stage_kernel<2, false><<<num_ctas, 256, 0, s>>>(K, iters, sink, cycles); break;
+        case 5: efq::stage_kernel<5, false><<<num_ctas, 256, 0, s>>>(K, iters, sink, cycles); break;
         case 4: efq::stage_kernel<4, false><<<num_ctas, 256, 0, s>>>(K, iters, sink, cycles); break;
         case 3: efq::stage_kernel<3, false><<<num_ctas, 256, 0, s>>>(efq::make_producer_consts_lut(0.08838834764831845f), iters, sink, cycles); break;
         default: return EFQ_ERR_INVALID_ARG;

@@ -15,7 +15,7 @@
 
 namespace efq {
 
-enum Producer : int { kEfq = 0, kEtq4 = 1, kEtq6 = 2, kEfqLut = 3, kEtq4Fold = 4 };
+enum Producer : int { kEfq = 0, kEtq4 = 1, kEtq6 = 2, kEfqLut = 3, kEtq4Fold = 4, kEtq4Hybrid = 5 };
 
 constexpr int kSegCols = 1024;       // columns per warp task
 constexpr int kWarpsPerCta = 8;
@@ -65,7 +65,7 @@ __device__ __forceinline__ void produce_block(const float (&r)[8], float m_s, co
         c -= (c >> 3) & 0x11111111u;        // floor(8w) = 8 only when v >= 8: that nibble is 7
         code32 = c;                         // a block without a finite score has w = 0 everywhere
         byte = s.byte;
-    } else if (PRODUCER == kEtq4Fold) {
+    } else if (PRODUCER == kEtq4Fold || PRODUCER == kEtq4Hybrid) {
         float rmax = fmaxf(max3(r[0], r[1], r[2]), max3(r[3], r[4], r[5]));
         rmax = max3(rmax, r[6], r[7]);
         rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, 1));
@@ -74,8 +74,9 @@ __device__ __forceinline__ void produce_block(const float (&r)[8], float m_s, co
         uint32_t c = 0;
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const float lo = ex2_approx(__fmaf_rn(r[2 * u], f.c1, f.c0e));
-            const float hi = ex2_approx(__fmaf_rn(r[2 * u + 1], f.c1, f.c0e));
+            const float tl = __fmaf_rn(r[2 * u], f.c1, f.c0e), th = __fmaf_rn(r[2 * u + 1], f.c1, f.c0e);
+            const float lo = (PRODUCER == kEtq4Hybrid && ex2_by_poly(2 * u)) ? ex2_poly3(tl) : ex2_approx(tl);
+            const float hi = (PRODUCER == kEtq4Hybrid && ex2_by_poly(2 * u + 1)) ? ex2_poly3(th) : ex2_approx(th);
             c |= (cvt_e2m1x2(lo, hi) & 0xffu) << (8 * u);
         }
         code32 = f.live ? c : 0u;
@@ -240,6 +241,7 @@ efq_status_t launch_probgen(int producer, const float* scores, int64_t ld, const
         case kEtq4: probgen_kernel<kEtq4><<<grid, block, 0, stream>>>(scores, ld, row_max, rows, cols, K, codes, scales, a32); break;
         case kEtq6: probgen_kernel<kEtq6><<<grid, block, 0, stream>>>(scores, ld, row_max, rows, cols, K, codes, scales, a32); break;
         case kEtq4Fold: probgen_kernel<kEtq4Fold><<<grid, block, 0, stream>>>(scores, ld, row_max, rows, cols, K, codes, scales, a32); break;
+        case kEtq4Hybrid: probgen_kernel<kEtq4Hybrid><<<grid, block, 0, stream>>>(scores, ld, row_max, rows, cols, K, codes, scales, a32); break;
         case kEfqLut: probgen_lut_kernel<<<grid, block, 0, stream>>>(scores, ld, row_max, rows, cols, K, codes, scales, a32); break;
         default: return EFQ_ERR_INVALID_ARG;
     }
@@ -268,7 +270,7 @@ extern "C" efq_status_t exp_then_quantize_probgen(const float* scores, int64_t l
                                                   int64_t rows, int64_t cols, float score_scale, int scale_mode,
                                                   uint8_t* codes, uint8_t* scales, void* stream)
 {
-    if (scale_mode < 0 || scale_mode > 2) return EFQ_ERR_INVALID_ARG;
-    return efq::launch_probgen(scale_mode == 0 ? efq::kEtq4 : scale_mode == 1 ? efq::kEtq6 : efq::kEtq4Fold, scores, ld, row_max, rows, cols,
+    if (scale_mode < 0 || scale_mode > 3) return EFQ_ERR_INVALID_ARG;
+    return efq::launch_probgen(scale_mode == 0 ? efq::kEtq4 : scale_mode == 1 ? efq::kEtq6 : scale_mode == 2 ? efq::kEtq4Fold : efq::kEtq4Hybrid, scores, ld, row_max, rows, cols,
                                score_scale, 0.0f, 1.0f, codes, scales, static_cast<cudaStream_t>(stream));
 }

@@ -185,7 +185,7 @@ def test_negative_threshold_is_refused():
     assert e.value.status == 1
 
 
-@pytest.mark.parametrize("mode,path", [(0, "etq"), (1, "etq6"), (2, "etq")])   # mode 2: mode 0 with the scale folded into ex2
+@pytest.mark.parametrize("mode,path", [(0, "etq"), (1, "etq6"), (2, "etq"), (3, "etq")])   # modes 2, 3: mode 0 with the scale folded into ex2 (3: part by polynomial)
 def test_exp_then_quantize_path(oracle, mode, path):
     case = inputs.AttentionCase("t", 1, 4, 2, 640, 640, 128, True, 9, "k_outliers")
     (q, k, v), (dq, dk, dv) = _case_tensors(case)

@@ -95,7 +95,7 @@ def test_probgen_unknown_variant_is_refused():
     assert e.value.status == 2
 
 
-@pytest.mark.parametrize("mode,name", [(0, "etq"), (1, "etq6"), (2, "etq")])   # mode 2: mode 0 with the scale folded into ex2
+@pytest.mark.parametrize("mode,name", [(0, "etq"), (1, "etq6"), (2, "etq"), (3, "etq")])   # modes 2, 3: mode 0 with the scale folded into ex2 (3: part by polynomial)
 def test_etq_probgen_statistical_parity(oracle, mode, name):
     scores, row_max = inputs.make_score_matrix(256, 4096 + 96, seed=7)
     scores[3, 100:300] = -np.inf
