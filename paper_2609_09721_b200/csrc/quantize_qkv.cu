@@ -57,11 +57,14 @@ __device__ __forceinline__ void mxfp4_block(const uint32_t (&w)[16], uint4& code
 __device__ __forceinline__ uint32_t sf_tile_offset(uint32_t r, uint32_t b) { return (r & 31u) * 16u + (r >> 5) * 4u + b; }
 
 // One thread per (row, 32-wide block along d); d = 128.  The input is addressed by strides in elements:
-// element (head, row, c) at x[head * head_stride + row * row_stride + c].
+// element (head, row, c) at x[head * head_stride + row * row_stride + c]; DENSE: rows of a head are contiguous
+// (row stride 128 known at compile time).
+template <bool DENSE>
 __global__ void __launch_bounds__(256)
 quantize_rows_kernel(const __nv_bfloat16* __restrict__ x, int64_t n_heads, int64_t S, int64_t S_pad,
-                     int64_t head_stride, int64_t row_stride, uint8_t* __restrict__ codes, uint8_t* __restrict__ sf)
+                     int64_t head_stride, int64_t row_stride_, uint8_t* __restrict__ codes, uint8_t* __restrict__ sf)
 {
+    const int64_t row_stride = DENSE ? 128 : row_stride_;
     const int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     const int64_t total = n_heads * S_pad * 4;
     if (t >= total) return;
@@ -87,10 +90,12 @@ quantize_rows_kernel(const __nv_bfloat16* __restrict__ x, int64_t n_heads, int64
 }
 
 // One thread per (32-key block, channel); consecutive threads take consecutive channels.
+template <bool DENSE>
 __global__ void __launch_bounds__(128)
 quantize_v_kernel(const __nv_bfloat16* __restrict__ v, int64_t n_heads, int64_t S, int64_t S_pad,
-                  int64_t head_stride, int64_t row_stride, uint8_t* __restrict__ vt_codes, uint8_t* __restrict__ sf)
+                  int64_t head_stride, int64_t row_stride_, uint8_t* __restrict__ vt_codes, uint8_t* __restrict__ sf)
 {
+    const int64_t row_stride = DENSE ? 128 : row_stride_;
     const int ch = threadIdx.x;                               // 0..127
     const int64_t kb = blockIdx.x;                            // key block over all heads
     const int64_t blocks_per_head = S_pad / 32;
@@ -118,8 +123,13 @@ cudaError_t launch_quantize_rows(const void* x, int64_t n_heads, int64_t S, int6
 {
     const int64_t total = n_heads * S_pad * 4;
     if (total == 0) return cudaSuccess;
-    quantize_rows_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, stream>>>(
-        static_cast<const __nv_bfloat16*>(x), n_heads, S, S_pad, head_stride, row_stride, codes, sf);
+    const unsigned grid = static_cast<unsigned>((total + 255) / 256);
+    if (row_stride == 128)
+        quantize_rows_kernel<true><<<grid, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(x), n_heads, S, S_pad,
+                                                            head_stride, row_stride, codes, sf);
+    else
+        quantize_rows_kernel<false><<<grid, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(x), n_heads, S, S_pad,
+                                                             head_stride, row_stride, codes, sf);
     return cudaGetLastError();
 }
 
@@ -128,8 +138,12 @@ cudaError_t launch_quantize_v(const void* v, int64_t n_heads, int64_t S, int64_t
 {
     const int64_t blocks = n_heads * (S_pad / 32);
     if (blocks == 0) return cudaSuccess;
-    quantize_v_kernel<<<static_cast<unsigned>(blocks), 128, 0, stream>>>(static_cast<const __nv_bfloat16*>(v), n_heads, S,
-                                                                         S_pad, head_stride, row_stride, vt_codes, sf);
+    if (row_stride == 128)
+        quantize_v_kernel<true><<<static_cast<unsigned>(blocks), 128, 0, stream>>>(
+            static_cast<const __nv_bfloat16*>(v), n_heads, S, S_pad, head_stride, row_stride, vt_codes, sf);
+    else
+        quantize_v_kernel<false><<<static_cast<unsigned>(blocks), 128, 0, stream>>>(
+            static_cast<const __nv_bfloat16*>(v), n_heads, S, S_pad, head_stride, row_stride, vt_codes, sf);
     return cudaGetLastError();
 }
 
