@@ -495,7 +495,7 @@ def run_cuda(args):
                 "api": "efq_attention_fwd_host_pipelined, %d chunks (KV heads), pinned host q/k/v in and fp32 o out every step" % n_chunks,
                 "single_stream_ms_per_step": e2e_plain_ms,
                 "single_stream_value": whole_job_tflops(flops, e2e_plain_ms, world)},
-        "gpu_launches": 4 * args.steps,
+        "gpu_launches": 2 * args.steps,     # operand preparation (one kernel for q, k, v) + fused forward
         "roofline": {"kernel": "attention_fwd_kernel<EFQ>", "bound": "tensor", "achieved": main_tflops, "peak": fp4_peak,
                      "unit": "TFLOP/s", "frac": main_tflops / fp4_peak, "traffic": traffic,
                      "peak_source": f"{peaks['source']} bf16 sustained {peaks['bf16_sustained']} TFLOP/s x {NOMINAL_FP4_OVER_BF16} "

@@ -171,7 +171,7 @@ efq_status_t efq_attention_fwd_quantized(float* o, int B, int Hq, int Hkv, int64
  * sequence sees its keys <= i + len_k - len_q, the rule of efq_attention_fwd); the operands of a sequence are
  * quantised by themselves, so the result of a sequence equals efq_attention_fwd on that sequence alone, bit for
  * bit.  A sequence without queries is skipped; one without keys gets zero rows.  `producer` as for
- * efq_attention_fwd_quantized.  The sequences are launched one after the other on `stream` (four kernels each)
+ * efq_attention_fwd_quantized.  The sequences are launched one after the other on `stream` (two kernels each)
  * and share one workspace slot: efq_attention_varlen_workspace_bytes() gives the size (0 for invalid arguments).
  * Asynchronous; efq_poll_status(workspace, stream) reports the first device-side problem of any sequence.
  * Errors: INVALID_ARG (null pointer, n_seqs < 0, prefix sums not starting at 0 or decreasing, bad params),

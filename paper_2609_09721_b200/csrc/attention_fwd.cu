@@ -36,10 +36,11 @@
 
 namespace efq {
 
-cudaError_t launch_quantize_rows(const void* x, int64_t n_heads, int64_t S, int64_t S_pad, int64_t head_stride,
-                                 int64_t row_stride, uint8_t* codes, uint8_t* sf, cudaStream_t stream);
-cudaError_t launch_quantize_v(const void* v, int64_t n_heads, int64_t S, int64_t S_pad, int64_t head_stride,
-                              int64_t row_stride, uint8_t* vt_codes, uint8_t* sf, cudaStream_t stream);
+cudaError_t launch_quantize_qkv(const void* q, const void* k, const void* v, int64_t q_heads, int64_t kv_heads, int64_t Sq,
+                                int64_t Sq_pad, int64_t Sk, int64_t Sk_pad, int64_t q_head_stride, int64_t q_row_stride,
+                                int64_t kv_head_stride, int64_t kv_row_stride, uint8_t* q_codes, uint8_t* q_sf,
+                                uint8_t* k_codes, uint8_t* k_sf, uint8_t* vt_codes, uint8_t* v_sf, uint32_t* status,
+                                cudaStream_t stream);
 
 namespace {
 
@@ -629,12 +630,13 @@ efq_status_t attention_impl(const void* q, const void* k, const void* v, float* 
 
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     if (do_quantize) {
-        if (cudaMemsetAsync(ws + w.status, 0, 1024, stream) != cudaSuccess) return EFQ_ERR_CUDA;
         const int64_t qh = token_major ? 128 : Sq * 128, qr = token_major ? static_cast<int64_t>(Hq) * 128 : 128;
         const int64_t kh = token_major ? 128 : Sk * 128, kr = token_major ? static_cast<int64_t>(Hkv) * 128 : 128;
-        if (launch_quantize_rows(q, static_cast<int64_t>(B) * Hq, Sq, w.Sq_pad, qh, qr, ws + w.qc, ws + w.qsf, stream) != cudaSuccess) return EFQ_ERR_CUDA;
-        if (launch_quantize_rows(k, static_cast<int64_t>(B) * Hkv, Sk, w.Sk_pad, kh, kr, ws + w.kc, ws + w.ksf, stream) != cudaSuccess) return EFQ_ERR_CUDA;
-        if (launch_quantize_v(v, static_cast<int64_t>(B) * Hkv, Sk, w.Sk_pad, kh, kr, ws + w.vt, ws + w.vsf, stream) != cudaSuccess) return EFQ_ERR_CUDA;
+        // one launch for the three operands; it also clears the status words the forward starts from
+        if (launch_quantize_qkv(q, k, v, static_cast<int64_t>(B) * Hq, static_cast<int64_t>(B) * Hkv, Sq, w.Sq_pad, Sk,
+                                w.Sk_pad, qh, qr, kh, kr, ws + w.qc, ws + w.qsf, ws + w.kc, ws + w.ksf, ws + w.vt,
+                                ws + w.vsf, reinterpret_cast<uint32_t*>(ws + w.status), stream) != cudaSuccess)
+            return EFQ_ERR_CUDA;
     }
     if (!do_forward) return EFQ_OK;
 
