@@ -589,3 +589,88 @@ def test_fp32_denominator_variant_of_the_baseline(oracle):
     ratio = p_q.sum(1) / p_f.sum(1)
     assert np.abs(o_fp - o_sh * ratio[:, None]).max() < 1e-5
     assert np.abs(ratio - 1.0).max() < 0.2 and np.abs(ratio - 1.0).max() > 1e-4
+
+
+# ---------------------------------------------------------------------------------------
+# causal alignment with Sq != Sk, and the ragged last block of the V quantiser
+# ---------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("Sq,Sk", [(100, 700), (260, 200)])
+def test_causal_mask_is_bottom_right_aligned_when_sq_differs_from_sk(oracle, Sq, Sk):
+    """Query i sees keys t <= i + Sk - Sq (the last query sees every key).  The exact path is compared with a
+    library softmax attention under that explicit boolean mask, so a top-left alignment (t <= i) fails; rows
+    that see no key (Sq > Sk, i < Sq - Sk) are zero; the dumped raw scores of the EFQ path are -inf exactly on
+    the masked keys."""
+    import torch
+    case = inputs.AttentionCase("t", 1, 4, 2, Sq, Sk, 128, True, 21, "iid")
+    q, k, v = (inputs.bf16_bits_to_f32(t) for t in inputs.make_qkv(case))
+    rows = np.array([(0, h, i) for h in range(4) for i in sorted({0, 1, Sq // 3, max(Sq - Sk, 0), Sq - 2, Sq - 1}
+                                                                 | set(range(5, Sq, 37)))], np.int64)
+    i_idx = torch.arange(Sq)[:, None]
+    t_idx = torch.arange(Sk)[None, :]
+    mask = t_idx <= i_idx + (Sk - Sq)
+    tq, tk, tv = (torch.from_numpy(t).double() for t in (q, k, v))
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        tq, tk.repeat_interleave(2, 1), tv.repeat_interleave(2, 1), attn_mask=mask, scale=case.softmax_scale).numpy()
+    out = oracle.attention_rows(q, k, v, rows, True, case.softmax_scale, "exact")
+    nvis = np.clip(rows[:, 2] + Sk - Sq + 1, 0, Sk)
+    seen = nvis > 0
+    assert seen.any() and (Sq <= Sk or (~seen).any())
+    want = ref[rows[:, 0], rows[:, 1], rows[:, 2]]
+    assert np.abs(out[seen] - want[seen]).max() < 1e-6
+    assert np.all(out[~seen] == 0.0)
+    for path in ("efq", "etq"):
+        o, d = oracle.attention_rows(q, k, v, rows, True, case.softmax_scale, path, dumps=True)
+        for n in range(rows.shape[0]):
+            assert np.all(np.isfinite(d["raw"][n, :nvis[n]])) and np.all(np.isneginf(d["raw"][n, nvis[n]:]))
+        assert np.all(o[~seen] == 0.0) and np.all(np.isfinite(o))
+        # a quantised path stays in the neighbourhood of the exact one only under the same alignment
+        rel = np.linalg.norm(o[seen] - out[seen]) / np.linalg.norm(out[seen])
+        assert rel < 0.5
+
+
+def test_v_quantiser_ragged_last_block_equals_zero_padded_block(oracle):
+    """88 keys = 2 full blocks + 24: the last block takes its maximum over the 24 valid keys only, which is what
+    quantising the matrix padded with zero rows to 96 keys gives (zeros change neither the maximum nor any code).
+    Checked against the padded column quantiser and against the row quantiser on the padded transpose."""
+    rng = np.random.default_rng(31)
+    v = (rng.normal(0, 1, (88, 128)) * np.exp2(rng.integers(-3, 4, (1, 128)))).astype(np.float32)
+    v = inputs.bf16_bits_to_f32(inputs.f32_to_bf16_bits(v))
+    v[64:, 5] = 0.0                                  # a channel whose ragged block is all zero: byte 0
+    v[87, 9] = 37.0                                  # the last valid key carries its block's maximum
+    vp = np.zeros((96, 128), np.float32)
+    vp[:88] = v
+    hat, codes, sc = oracle.mxfp4_cols(v)
+    hat_p, codes_p, sc_p = oracle.mxfp4_cols(vp)
+    assert np.array_equal(hat, hat_p[:88]) and np.array_equal(codes, codes_p[:88]) and np.array_equal(sc, sc_p)
+    rhat, rcodes, rsc = oracle.mxfp4_rows(np.ascontiguousarray(vp.T))       # blocks of 32 along the padded keys
+    assert np.array_equal(hat, rhat.T[:88]) and np.array_equal(codes, rcodes.T[:88]) and np.array_equal(sc, rsc.T)
+    assert sc[2, 5] == 0 and np.all(hat[64:, 5] == 0.0)
+    assert sc[2, 9] == 127 + 3 and hat[87, 9] == 32.0     # 37 = 4.625 * 2^3 -> nearest code 4: the last key is really quantised
+
+
+@pytest.mark.parametrize("path", ["efq", "etq", "efq_lut"])
+def test_attention_with_ragged_key_count_matches_closed_form(oracle, path):
+    """Sk = 88 (one KV tile, last block of 24 keys): O rebuilt from the dumped operand and a V dequantised through
+    the zero-padded matrix - (P~ V^) / (P~ 1) - so a key dropped from the ragged block, in the value quantiser or
+    in the producer, shows."""
+    case = inputs.AttentionCase("t", 1, 4, 2, 88, 88, 128, False, 33, "iid")
+    q, k, v = (inputs.bf16_bits_to_f32(t) for t in inputs.make_qkv(case))
+    rows = np.array([(0, h, i) for h in range(4) for i in range(0, 88, 5)], np.int64)
+    out, d = oracle.attention_rows(q, k, v, rows, False, case.softmax_scale, path, Bc=128, dumps=True)
+    codes = oracle.unpack_codes(d["codes"])[:, :88].astype(np.int64)
+    kexp = d["scales"].astype(np.int64) - 127
+    assert kexp.shape[1] == 3
+    p = efq_math.dequant_probabilities(np.pad(codes, ((0, 0), (0, 8))), kexp)[:, :88]
+    assert np.all(p[:, 87] >= 0) and (p[:, 64:] > 0).any()
+    for n, (b, h, i) in enumerate(rows):
+        vp = np.zeros((96, 128), np.float32)
+        vp[:88] = v[b, h // 2]
+        vhat = oracle.mxfp4_rows(np.ascontiguousarray(vp.T))[0].T[:88]
+        want = efq_math.attention_from_operand(p[n:n + 1], vhat)[0]
+        assert np.abs(out[n] - want).max() < 1e-6
+    # the block maximum of the ragged block is over its 24 valid keys: top code region, never a masked key
+    if path == "efq":
+        x = d["raw"][:, 64:88].astype(np.float64)
+        top = codes[:, 64:88][np.arange(rows.shape[0]), x.argmax(1)]
+        assert np.all(top == 7)
