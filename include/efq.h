@@ -120,7 +120,8 @@ efq_status_t exp_then_quantize_probgen(const float* scores, int64_t ld, const fl
                                        uint8_t* scales, void* stream);
 
 /* Bytes of caller-owned device workspace the fused forward needs for a problem shape
- * (MXFP4 copies of Q, K, V with their scale tensors, tensor-map descriptors, status word).
+ * (MXFP4 copies of Q, K, V with their scale tiles, and the status word; tensor-map descriptors are built on the
+ * host and travel as kernel parameters).
  * Returns 0 for an unsupported shape. */
 size_t efq_attention_workspace_bytes(int B, int Hq, int Hkv, int64_t Sq, int64_t Sk, int d);
 
@@ -202,7 +203,10 @@ efq_status_t efq_attention_fwd_host(const void* q_host, const void* k_host, cons
  * problem does whenever two or more chunks are used (with a single chunk the call is efq_attention_fwd_host on
  * `stream_compute`).  The call is asynchronous; when the work queued on
  * `stream_compute` has completed, so have the last copies, and efq_poll_status(workspace, stream_compute) reports
- * a device-side timeout of any chunk.  Errors as efq_attention_fwd_host, plus INVALID_ARG for n_chunks <= 0. */
+ * a device-side timeout of any chunk.  Calls may follow one another with the same staging buffers and workspace:
+ * at entry `stream_in` is made to wait for the work `stream_compute` already holds, so the input copies of a call
+ * never overtake the forwards of the call before it.  (The host output buffer of the earlier call is complete once
+ * `stream_compute` has been synchronised.)  Errors as efq_attention_fwd_host, plus INVALID_ARG for n_chunks <= 0. */
 efq_status_t efq_attention_fwd_host_pipelined(const void* q_host, const void* k_host, const void* v_host, float* o_host,
                                               void* q_dev, void* k_dev, void* v_dev, float* o_dev, int B, int Hq,
                                               int Hkv, int64_t Sq, int64_t Sk, int d, int causal, float softmax_scale,

@@ -455,7 +455,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 
             // The registers are free: if S of the group's next tile is there already (it is as a rule, S runs ahead),
             // its scores set out now and travel while the operand is handed over and the loop turns.
-            in_flight = !DEBUG && j + 2 < n_tiles && ptx::mbar_try_wait(&sm->s_full[sb], ph2 ^ 1u);
+            in_flight = j + 2 < n_tiles && ptx::mbar_try_wait(&sm->s_full[sb], ph2 ^ 1u);
             if (in_flight) {
                 ptx::tc_fence_after_sync();
                 ptx::tmem_ld32f<0>(s_addr, r);
@@ -518,31 +518,61 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+constexpr int kMaxDevices = 64;   // device ordinals the per-device tables of this file cover
+
 EncodeTiledFn get_encode()
 {
+    static std::once_flag once;
     static EncodeTiledFn fn = nullptr;
-    if (!fn) {
+    std::call_once(once, [] {
         void* p = nullptr;
         cudaDriverEntryPointQueryResult q;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
             q == cudaDriverEntryPointSuccess)
             fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
+    });
     return fn;
 }
 
-// [rows, row_bytes] u8 matrix, box 64 B x 128 rows, 64-byte swizzle
+// [rows, row_bytes] u8 matrix, box 64 B x 128 rows, 64-byte swizzle.  A descriptor depends on nothing but
+// (base, row_bytes, rows), so the last few are kept: a serving loop that calls with the same workspace and shape
+// (decode steps above all) does not pay for three driver calls per forward.
+struct MapCacheEntry {
+    const void* base;
+    uint64_t row_bytes, rows;
+    CUtensorMap map;
+};
+constexpr int kMapCacheSize = 24;
+std::mutex g_map_mutex;
+MapCacheEntry g_map_cache[kMapCacheSize] = {};
+int g_map_next = 0;
+
 bool encode_map(CUtensorMap* map, const void* base, uint64_t row_bytes, uint64_t rows)
 {
+    {
+        std::lock_guard<std::mutex> lock(g_map_mutex);
+        for (int i = 0; i < kMapCacheSize; ++i) {
+            const MapCacheEntry& e = g_map_cache[i];
+            if (e.base == base && e.row_bytes == row_bytes && e.rows == rows) {
+                *map = e.map;
+                return true;
+            }
+        }
+    }
     EncodeTiledFn enc = get_encode();
     if (!enc) return false;
     cuuint64_t dims[2] = {row_bytes, rows};
     cuuint64_t strides[1] = {row_bytes};
     cuuint32_t box[2] = {64, 128};
     cuuint32_t estr[2] = {1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    if (enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return false;
+    std::lock_guard<std::mutex> lock(g_map_mutex);
+    g_map_cache[g_map_next] = MapCacheEntry{base, row_bytes, rows, *map};
+    g_map_next = (g_map_next + 1) % kMapCacheSize;
+    return true;
 }
 
 struct Workspace {
@@ -580,9 +610,20 @@ template <int PRODUCER, bool DEBUG, bool FIX8>
 cudaError_t launch_one(dim3 grid, size_t smem, cudaStream_t stream, const CUtensorMap& mq, const CUtensorMap& mk,
                        const CUtensorMap& mv, const FwdParams& P)
 {
-    cudaError_t e = cudaFuncSetAttribute(attention_fwd_kernel<PRODUCER, DEBUG, FIX8>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-    if (e != cudaSuccess) return e;
+    // the shared-memory attribute belongs to (function, device): set once for each
+    static std::mutex mu;
+    static bool done[kMaxDevices] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (!done[dev]) {
+            cudaError_t e = cudaFuncSetAttribute(attention_fwd_kernel<PRODUCER, DEBUG, FIX8>,
+                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+            if (e != cudaSuccess) return e;
+            done[dev] = true;
+        }
+    }
     attention_fwd_kernel<PRODUCER, DEBUG, FIX8><<<grid, kThreads, smem, stream>>>(mq, mk, mv, P);
     return cudaGetLastError();
 }
@@ -841,6 +882,12 @@ extern "C" efq_status_t efq_attention_fwd_host_pipelined(const void* q_host, con
     const size_t o_head = static_cast<size_t>(Sq) * d * 4;
     cudaEvent_t ev = nullptr;
     auto fail = [&](efq_status_t code) { if (ev) cudaEventDestroy(ev); return code; };
+    // The staging buffers are reused from call to call: this call's input copies must not overtake the forwards
+    // of an earlier call that still read them, so stream_in first waits for what stream_compute holds now.
+    if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess) return EFQ_ERR_CUDA;
+    if (cudaEventRecord(ev, s_c) != cudaSuccess || cudaStreamWaitEvent(s_in, ev, 0) != cudaSuccess) return fail(EFQ_ERR_CUDA);
+    cudaEventDestroy(ev);
+    ev = nullptr;
     for (int b = 0; b < B; ++b) {
         for (int h0 = 0; h0 < Hkv; h0 += heads_per_chunk) {
             const int nh = h0 + heads_per_chunk <= Hkv ? heads_per_chunk : Hkv - h0;
@@ -985,7 +1032,7 @@ static __device__ __align__(256) uint8_t g_static_scratch[EFQ_STATIC_SCRATCH_BYT
 
 namespace {
 
-constexpr int kMaxDevices = 64;
+constexpr int kMaxDevices = 64;   // device ordinals this table covers
 std::mutex g_static_mutex;
 void* g_static_ptr[kMaxDevices] = {};   // device address of g_static_scratch, per device ordinal
 
@@ -1016,7 +1063,9 @@ extern "C" efq_status_t efq_attention_fwd_static(const void* q, const void* k, c
     bool lut;
     efq_status_t st;
     if (!read_params(params, tau, h, lut, threshold, st)) return st;
-    if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0) return EFQ_ERR_INVALID_ARG;
+    // the argument rules of efq_attention_fwd, in its order, before the size of the problem is looked at
+    if (!q || !k || !v || !o) return EFQ_ERR_INVALID_ARG;
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0 || Hq % Hkv != 0) return EFQ_ERR_INVALID_ARG;
     if (d != 128) return EFQ_ERR_UNSUPPORTED;
     const size_t need = efq_attention_workspace_bytes(B, Hq, Hkv, Sq, Sk, d);
     if (need == 0) return EFQ_ERR_UNSUPPORTED;

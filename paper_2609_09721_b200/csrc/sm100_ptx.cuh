@@ -55,6 +55,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
         : "memory");
     return done != 0;
 }
+// Non-blocking test of a phase: never suspends the thread.  (try_wait may hold the thread for an implementation-
+// defined time when the phase is still pending, so a poll placed ahead of useful work must use this form.)
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity)
+{
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}\n"
+        : "=r"(done)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return done != 0;
+}
 // Same test, but the thread may stay suspended in hardware for up to `ns` nanoseconds while the phase is
 // pending, instead of returning to a polling loop that would take issue slots from the compute warps.
 __device__ __forceinline__ bool mbar_try_wait_suspend(uint64_t* bar, uint32_t parity, uint32_t ns)

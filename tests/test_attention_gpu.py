@@ -88,6 +88,11 @@ def test_single_head_1024_full_dump(oracle, params):
     assert np.array_equal(dump.scales.cpu().numpy(), want["scales"])
     got = o.cpu().numpy()[0, 0]
     assert np.abs(got - want_o).max() <= TOL_O
+    # the instantiation without the dump - the one that is timed - gives the same output bit for bit, so the
+    # bit-exact operand check above holds for it too
+    o_prod = binding.efq_attention_fwd(dq, dk, dv, False, 0.0, params)
+    torch.cuda.synchronize()
+    assert torch.equal(o, o_prod)
     exact = oracle.attention_rows(q, k, v, rows, False, case.softmax_scale, "exact")
     print("single_head_1024: max|O_gpu-O_oracle| =", np.abs(got - want_o).max(),
           " rel-Frobenius vs exact =", np.linalg.norm(got - exact) / np.linalg.norm(exact))
@@ -109,6 +114,23 @@ def test_small_shapes_efq(oracle, S, Hq, Hkv, causal, recipe):
     got = o.cpu().numpy().reshape(-1, 128)
     assert np.abs(got - want_o).max() <= TOL_O
     _check_dump(oracle, case, dump, _all_rows(case, head, 0, S), MEAN)
+    o_prod = binding.efq_attention_fwd(dq, dk, dv, causal, 0.0, None)     # production instantiation: same bits
+    torch.cuda.synchronize()
+    assert torch.equal(o, o_prod)
+
+
+def test_production_kernel_equals_dumped_kernel_on_a_long_causal_gqa_case(oracle):
+    """S = 2048 (16 KV tiles: every role's steady state, prefetch of the next scores included), causal, GQA, K
+    outliers: the dump of one head is bit-exact against the oracle and the kernel without the dump returns the same
+    output for every head, so the timed instantiation is tied to the bit-exact check by an equality."""
+    case = inputs.AttentionCase("prod", 1, 8, 2, 2048, 2048, 128, True, 97, "k_outliers")
+    (q, k, v), (dq, dk, dv) = _case_tensors(case)
+    dump = binding.DebugDump(0, 5, 1024, 2048, 2048)
+    o = binding.efq_attention_fwd(dq, dk, dv, True, 0.0, None, debug=dump)
+    o_prod = binding.efq_attention_fwd(dq, dk, dv, True, 0.0, None)
+    torch.cuda.synchronize()
+    assert torch.equal(o, o_prod)
+    _check_dump(oracle, case, dump, _all_rows(case, 5, 1024, 2048), MEAN)
 
 
 @pytest.mark.parametrize("Sq,Sk,causal", [(128, 512, True), (100, 700, False), (260, 200, True), (64, 4096 + 88, True),

@@ -11,8 +11,6 @@ from paper_2609_09721_b200 import binding, inputs
 
 pytestmark = pytest.mark.gpu
 
-TOL_O = 2e-3
-
 
 def _dev(bits):
     return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
@@ -33,7 +31,7 @@ def test_static_scratch_forward_matches_workspace_forward_twice():
         assert torch.cuda.memory_stats()["allocation.all.allocated"] == before   # no request reached torch's allocator either
         assert got.data_ptr() == o.data_ptr()
         assert torch.isfinite(got).all()
-        assert (got - want).abs().max().item() <= TOL_O
+        assert torch.equal(got, want)       # the same kernels on the same operands: not a tolerance, the same bits
     # same problem again, back to back: results repeat exactly
     again = binding.efq_attention_fwd_static(q, k, v, case.causal, o=torch.empty_like(want))
     torch.cuda.synchronize()
@@ -48,3 +46,11 @@ def test_static_scratch_limit_is_reported():
         binding.efq_attention_fwd_static(q, q, q, True, o=torch.empty((1, 8, S, 128), dtype=torch.float32, device="cuda"))
     assert e.value.status == binding.STATUS_NAMES.index("EFQ_ERR_STATIC_LIMIT")
     assert "built-in scratch" in str(e.value)
+
+
+def test_static_entry_applies_the_argument_rules_of_the_regular_forward():
+    q = torch.zeros((1, 3, 128, 128), dtype=torch.bfloat16, device="cuda")
+    k = torch.zeros((1, 2, 128, 128), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(binding.EfqError) as e:       # Hq % Hkv != 0 is an invalid argument here too
+        binding.efq_attention_fwd_static(q, k, k, False, o=torch.empty((1, 3, 128, 128), dtype=torch.float32, device="cuda"))
+    assert e.value.status == binding.STATUS_NAMES.index("EFQ_ERR_INVALID_ARG")
