@@ -36,9 +36,13 @@ UNIT = "TFLOP/s"
 NOMINAL_FP4_OVER_BF16 = 4.0          # dense FP4 : dense bf16 tensor throughput on B200 (9 : 2.25 PFLOP/s)
 FALLBACK_BF16_TFLOPS = 1590.0
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the fused kernel, from the ncu capture summarised in
-# profiles/attention_fwd_qwen3_8b_16k.md (a single-pass capture at full size)
-NCU_DRAM_BYTES_PER_LAUNCH = {"qwen3_8b_16k": 57208832 + 217094144}
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the fused kernel: NOT measured by this run, copied
+# from the single-pass ncu capture summarised in the named profile, and valid only for the kernel revision that
+# capture saw (the library's version tag); for any other revision the line carries null.
+NCU_DRAM_BYTES_PER_LAUNCH = {
+    "qwen3_8b_16k": {"bytes": 57208832 + 217094144, "kernel_revision": "fwd.3", "profile": "profiles/attention_fwd_qwen3_8b_16k.md"},
+}
+BURST_REGION_S = 1.0   # a timed region shorter than this runs at burst clocks: its roofline uses the burst peak
 
 
 def workload_case(name: str) -> inputs.AttentionCase:
@@ -274,14 +278,12 @@ def run_cuda(args):
     dev = torch.device("cuda", local_rank)
     binding.lib()
 
-    case = workload_case(args.workload)
-    qb, kb, vb = inputs.make_qkv(case)     # every rank: its own replica of the workload (weak scaling, no exchange)
-    pin = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).pin_memory()
-    hq, hk, hv = pin(qb), pin(kb), pin(vb)
-    dq, dk, dv = hq.to(dev), hk.to(dev), hv.to(dev)
-    shape = (case.B, case.Hq, case.Hkv, case.Sq, case.Sk, case.d)
-    o = torch.empty((case.B, case.Hq, case.Sq, case.d), dtype=torch.float32, device=dev)
-    ws = torch.empty(binding.efq_attention_workspace_bytes(*shape), dtype=torch.uint8, device=dev)
+    LUT = (0.0, 1.0, 1)      # efq_params_t with variant 1: the EFQ-Softmax-LUT ablation (tau, h not read)
+    LAZY = (-3.06, 2.30, 0, 0, 4.0)   # EFQ-Mean with the optional thresholded rescaling (T = 4 scaled units; not in the paper)
+    # timed variants: the library's producer id (0 EFQ, 1 exp-then-quantize, 4 the same with the scale folded into ex2,
+    # 6 exp-then-quantize whose denominator is the sum of the FP32 exponentials) and the efq_params_t that goes with it
+    VARIANTS = {"efq": (0, None), "etq": (1, None), "etq_folded": (4, None), "etq_hybrid": (5, None), "efq_lut": (0, LUT),
+                "efq_lazy": (0, LAZY), "etq_fp32den": (6, None)}
     stream = torch.cuda.current_stream()
 
     def barrier():
@@ -289,43 +291,59 @@ def run_cuda(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    LUT = (0.0, 1.0, 1)      # efq_params_t with variant 1: the EFQ-Softmax-LUT ablation (tau, h not read)
-    LAZY = (-3.06, 2.30, 0, 0, 4.0)   # EFQ-Mean with the optional thresholded rescaling (T = 4 scaled units; not in the paper)
+    class Workload:
+        """Device-resident inputs, output and workspace of one attention configuration."""
 
-    # timed variants: the library's producer id (0 EFQ, 1 exp-then-quantize, 4 the same with the scale folded into ex2)
-    # and the efq_params_t that goes with it
-    VARIANTS = {"efq": (0, None), "etq": (1, None), "etq_folded": (4, None), "etq_hybrid": (5, None), "efq_lut": (0, LUT), "efq_lazy": (0, LAZY)}
+        def __init__(self, name):
+            self.case = workload_case(name)
+            case = self.case
+            self.qb, self.kb, self.vb = inputs.make_qkv(case)   # every rank: its own replica (weak scaling, no exchange)
+            pin = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16).pin_memory()
+            self.hq, self.hk, self.hv = pin(self.qb), pin(self.kb), pin(self.vb)
+            self.dq, self.dk, self.dv = self.hq.to(dev), self.hk.to(dev), self.hv.to(dev)
+            self.shape = (case.B, case.Hq, case.Hkv, case.Sq, case.Sk, case.d)
+            self.o = torch.empty((case.B, case.Hq, case.Sq, case.d), dtype=torch.float32, device=dev)
+            self.ws = torch.empty(binding.efq_attention_workspace_bytes(*self.shape), dtype=torch.uint8, device=dev)
 
-    def step(variant="efq", ev=None):
-        producer, prm = VARIANTS[variant]
-        binding.efq_quantize_qkv(dq, dk, dv, ws)
-        if ev is not None:
-            ev[0].record(stream)
-        binding.efq_attention_fwd_quantized(o, shape, ws, case.causal, 0.0, producer, prm)
-        if ev is not None:
-            ev[1].record(stream)
+        def step(self, variant="efq", ev=None):
+            producer, prm = VARIANTS[variant]
+            binding.efq_quantize_qkv(self.dq, self.dk, self.dv, self.ws)
+            if ev is not None:
+                ev[0].record(stream)
+            binding.efq_attention_fwd_quantized(self.o, self.shape, self.ws, self.case.causal, 0.0, producer, prm)
+            if ev is not None:
+                ev[1].record(stream)
 
-    def timed(producer, steps, warmup, sampler=None):
-        for _ in range(warmup):
-            step(producer)
-        barrier()
-        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        if sampler:
-            sampler.start()
-            time.sleep(0.25)
-        t0 = time.time()
-        e0.record(stream)
-        for i in range(steps):
-            step(producer, evs[i])
-        e1.record(stream)
-        barrier()
-        t1 = time.time()
-        clocks = sampler.stop(t0, t1) if sampler else None
-        ms = e0.elapsed_time(e1)
-        main_ms = sum(a.elapsed_time(b) for a, b in evs) / steps
-        ms, main_ms = max_over_ranks([ms, main_ms], dev)
-        return ms / steps, main_ms, clocks
+        def timed(self, variant, steps, warmup, sampler=None):
+            """(ms per step, ms of the fused kernel per launch, clocks): CUDA events on the launching stream, the
+            slowest rank's figures."""
+            for _ in range(warmup):
+                self.step(variant)
+            barrier()
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            if sampler:
+                sampler.start()
+                time.sleep(0.25)
+            t0 = time.time()
+            e0.record(stream)
+            for i in range(steps):
+                self.step(variant, evs[i])
+            e1.record(stream)
+            barrier()
+            t1 = time.time()
+            clocks = sampler.stop(t0, t1) if sampler else None
+            ms = e0.elapsed_time(e1)
+            main_ms = sum(a.elapsed_time(b) for a, b in evs) / steps
+            ms, main_ms = max_over_ranks([ms, main_ms], dev)
+            if binding.efq_poll_status(self.ws) != 0:
+                raise SystemExit(f"bench.py: device status set after timing {variant} on {self.case.name}")
+            return ms / steps, main_ms, clocks
+
+    wl = Workload(args.workload)
+    case, qb, kb, vb = wl.case, wl.qb, wl.kb, wl.vb
+    hq, hk, hv, dq, dk, dv, shape, o, ws = wl.hq, wl.hk, wl.hv, wl.dq, wl.dk, wl.dv, wl.shape, wl.o, wl.ws
+    timed = wl.timed
 
     phys_gpu = local_rank
     vis = os.environ.get("CUDA_VISIBLE_DEVICES")
@@ -336,10 +354,8 @@ def run_cuda(args):
             phys_gpu = local_rank
     sampler = ClockSampler(phys_gpu) if rank == 0 else None
     ms_step, ms_main, clocks = timed("efq", args.steps, args.warmup, sampler)
-    status = binding.efq_poll_status(ws)
-    if status != 0:
-        raise SystemExit(f"bench.py: device status {status} after the timed region")
     etq_ms_step, etq_ms_main, _ = timed("etq", max(3, args.steps // 2), 3)
+    etqd_ms_step, etqd_ms_main, _ = timed("etq_fp32den", max(3, args.steps // 2), 3)
     etqf_ms_step, etqf_ms_main, _ = timed("etq_folded", max(3, args.steps // 2), 3)
     etqh_ms_step, etqh_ms_main, _ = timed("etq_hybrid", max(3, args.steps // 2), 3)
     lut_ms_step, lut_ms_main, _ = timed("efq_lut", max(3, args.steps // 4), 3)
@@ -383,38 +399,50 @@ def run_cuda(args):
     if binding.efq_poll_status(ws) != 0:
         raise SystemExit("bench.py: device status set after the end-to-end region")
 
-    # standalone probability-generation stage (HBM-bound): EFQ vs exp-then-quantize, 4096 x 16384 fp32
+    # standalone probability-generation stage (HBM-bound): EFQ vs exp-then-quantize on the stage configuration
+    # (fp32 4096 x 16384, N(0, 9) with a seeded 1 % of each row set to +12, row maximum precomputed), two buffer sets
+    # used in turn so that no launch finds its input or output lines in L2 (each set is 304 MB of traffic anyway)
     stage = None
     if rank == 0 and not args.skip_stage:
         rows, cols = 4096, 16384
-        g = torch.Generator(device=dev)
-        g.manual_seed(2)
-        sc = torch.randn((rows, cols), generator=g, device=dev, dtype=torch.float32) * 3.0
-        rm = sc.max(dim=1).values.contiguous()
-        codes = torch.empty((rows, cols // 2), dtype=torch.uint8, device=dev)
-        scl = torch.empty((rows, cols // 32), dtype=torch.uint8, device=dev)
+        h_sc, h_rm = inputs.make_score_matrix(rows, cols, seed=2)
+        sets = []
+        for shift in (0, 1):          # second set: the same rows one place further on (same statistics, other addresses)
+            sc = torch.from_numpy(np.roll(h_sc, shift, axis=0)).to(dev)
+            rm = torch.from_numpy(np.roll(h_rm, shift, axis=0)).to(dev)
+            sets.append((sc, rm, torch.empty((rows, cols // 2), dtype=torch.uint8, device=dev),
+                         torch.empty((rows, cols // 32), dtype=torch.uint8, device=dev)))
+        del h_sc, h_rm
         nbytes = rows * cols * (4 + 0.5 + 1 / 32)
+        n_stage = 20
 
         def stage_time(fn):
-            for _ in range(3):
-                fn()
+            for i in range(4):
+                fn(*sets[i & 1])
             torch.cuda.synchronize()
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record(stream)
-            for _ in range(20):
-                fn()
+            for i in range(n_stage):
+                fn(*sets[i & 1])
             b.record(stream)
             torch.cuda.synchronize()
-            return a.elapsed_time(b) / 20
+            return a.elapsed_time(b) / n_stage
 
-        t_efq = stage_time(lambda: binding.efq_probgen(sc, rm, 1.0, None, codes, scl))
-        t_etq = stage_time(lambda: binding.exp_then_quantize_probgen(sc, rm, 1.0, 0, codes, scl))
-        t_etqf = stage_time(lambda: binding.exp_then_quantize_probgen(sc, rm, 1.0, 2, codes, scl))
-        t_etqh = stage_time(lambda: binding.exp_then_quantize_probgen(sc, rm, 1.0, 3, codes, scl))
-        t_lut = stage_time(lambda: binding.efq_probgen(sc, rm, 1.0, LUT, codes, scl))
-        stage = {"workload": "probgen 4096x16384 fp32 (device-generated N(0,9), timing only)", "bytes_per_launch": nbytes,
-                 "efq_ms": t_efq, "efq_gbs": nbytes / t_efq / 1e6, "etq_ms": t_etq, "etq_gbs": nbytes / t_etq / 1e6,
-                 "etq_folded_ms": t_etqf, "etq_folded_gbs": nbytes / t_etqf / 1e6, "etq_hybrid_ms": t_etqh, "etq_hybrid_gbs": nbytes / t_etqh / 1e6, "efq_lut_ms": t_lut, "efq_lut_gbs": nbytes / t_lut / 1e6}
+        t_efq = stage_time(lambda sc, rm, c, sl: binding.efq_probgen(sc, rm, 1.0, None, c, sl))
+        t_etq = stage_time(lambda sc, rm, c, sl: binding.exp_then_quantize_probgen(sc, rm, 1.0, 0, c, sl))
+        t_etqf = stage_time(lambda sc, rm, c, sl: binding.exp_then_quantize_probgen(sc, rm, 1.0, 2, c, sl))
+        t_etqh = stage_time(lambda sc, rm, c, sl: binding.exp_then_quantize_probgen(sc, rm, 1.0, 3, c, sl))
+        t_lut = stage_time(lambda sc, rm, c, sl: binding.efq_probgen(sc, rm, 1.0, LUT, c, sl))
+        hbm = measured_peaks()["hbm_gbs"]
+        stage = {"workload": "probgen 4096x16384 fp32, N(0,9) with 1 % of each row at +12 (seed 2), 2 buffer sets in turn",
+                 "bytes_per_launch": nbytes, "launches_timed": n_stage, "hbm_peak_gbs": hbm,
+                 "bound": "hbm: both producers sit on the bandwidth line in wall time; they separate in the in-SM rate "
+                          "(microbench) and in the fused forward",
+                 "efq_ms": t_efq, "efq_gbs": nbytes / t_efq / 1e6, "efq_frac_of_hbm_peak": nbytes / t_efq / 1e6 / hbm,
+                 "etq_ms": t_etq, "etq_gbs": nbytes / t_etq / 1e6, "etq_frac_of_hbm_peak": nbytes / t_etq / 1e6 / hbm,
+                 "etq_folded_ms": t_etqf, "etq_folded_gbs": nbytes / t_etqf / 1e6, "etq_hybrid_ms": t_etqh,
+                 "etq_hybrid_gbs": nbytes / t_etqh / 1e6, "efq_lut_ms": t_lut, "efq_lut_gbs": nbytes / t_lut / 1e6}
+        del sets
 
     # accuracy beside the speed: relative Frobenius error of each producer's output against FP32 attention on
     # the unquantised inputs, on the whole benchmarked problem (reference kernel: plain CUDA cores, run once)
@@ -429,6 +457,7 @@ def run_cuda(args):
         binding.efq_quantize_qkv(dq, dk, dv, ws)
         for name, prod, prm in (("efq", 0, None), ("exp_then_quantize", 1, None), ("exp_then_quantize_scale6", 2, None),
                                 ("exp_then_quantize_folded", 4, None), ("exp_then_quantize_hybrid", 5, None),
+                                ("exp_then_quantize_fp32_denominator", 6, None),
                                 ("efq_lut", 0, LUT), ("efq_mmlu", 0, (-2.90, 2.00)), ("efq_balance", 0, (-2.10, 2.70)),
                                 ("efq_thresholded_rescale_T4", 0, LAZY)):
             binding.efq_attention_fwd_quantized(o, shape, ws, case.causal, 0.0, prod, prm)
@@ -470,9 +499,55 @@ def run_cuda(args):
     peaks = measured_peaks()
     flops = case.flops
     value = whole_job_tflops(flops, ms_step, world)
-    main_tflops = flops / (ms_main * 1e-3) / 1e12
-    fp4_peak = peaks["bf16_sustained"] * NOMINAL_FP4_OVER_BF16
-    traffic = NCU_DRAM_BYTES_PER_LAUNCH.get(args.workload)
+    mma_only = micro["fp4_mma_only_tflops"] if micro else None
+
+    def roofline_of(flops_per_launch, ms_launch, region_s, workload_name):
+        """Roofline object of the fused kernel: achieved = algorithmic FLOPs of a launch / its CUDA-event duration; the
+        peak is the measured cuBLAS bf16 rate x 4 (nominal FP4 : bf16), the burst figure for a timed region under
+        BURST_REGION_S and the sustained one above it; the other denominators are given beside it."""
+        achieved = flops_per_launch / (ms_launch * 1e-3) / 1e12
+        burst = region_s < BURST_REGION_S
+        bf16 = peaks["bf16_burst"] if burst else peaks["bf16_sustained"]
+        peak = bf16 * NOMINAL_FP4_OVER_BF16
+        entry = NCU_DRAM_BYTES_PER_LAUNCH.get(workload_name)
+        traffic, traffic_source = None, None
+        if entry is not None:
+            if entry["kernel_revision"] in binding.version():
+                traffic = entry["bytes"]
+                traffic_source = f"not measured by this run: ncu capture of kernel revision {entry['kernel_revision']}, {entry['profile']}"
+            else:
+                traffic_source = f"dropped: the ncu capture in {entry['profile']} saw kernel revision {entry['kernel_revision']}, this library is {binding.version()}"
+        return {"kernel": "attention_fwd_kernel<EFQ>", "bound": "tensor", "achieved": achieved, "peak": peak,
+                "unit": "TFLOP/s", "frac": achieved / peak, "traffic": traffic, "traffic_source": traffic_source,
+                "peak_source": f"{peaks['source']} bf16 {'burst' if burst else 'sustained'} {bf16} TFLOP/s x {NOMINAL_FP4_OVER_BF16} "
+                               f"(nominal FP4:bf16 ratio); timed region {region_s:.3f} s",
+                "ms_per_launch": ms_launch,
+                "frac_of_bf16_burst_x4": achieved / (peaks["bf16_burst"] * NOMINAL_FP4_OVER_BF16),
+                "frac_of_bf16_sustained_x4": achieved / (peaks["bf16_sustained"] * NOMINAL_FP4_OVER_BF16),
+                "frac_of_fp4_mma_only_probe": achieved / mma_only if mma_only else None,
+                "frac_of_nominal_9pflops": achieved / 9000.0}
+
+    roofline = roofline_of(flops, ms_main, ms_step * args.steps * 1e-3, args.workload)
+
+    # the other two attention shapes of the metric, a few steps each (EFQ and the strongest exponential baseline),
+    # with their own step time, roofline fraction and clocks
+    others = None
+    if world == 1 and not args.skip_other_workloads:
+        others = {}
+        for name in [n for n in ("wan22_32760", "qwen3_8b_128k") if n != args.workload]:
+            w2 = Workload(name)
+            n2 = 5
+            ms2, main2, clk2 = w2.timed("efq", n2, 3, ClockSampler(phys_gpu))
+            f_ms2, f_main2, _ = w2.timed("etq_folded", 3, 3)
+            c2 = w2.case
+            others[name] = {"config": {"workload": c2.name, "B": c2.B, "Hq": c2.Hq, "Hkv": c2.Hkv, "S": c2.Sq, "d": c2.d,
+                                       "causal": c2.causal, "kv_tile": 128},
+                            "steps": n2, "warmup": 3, "ms_per_step": ms2, "value": c2.flops / (ms2 * 1e-3) / 1e12, "unit": UNIT,
+                            "roofline": roofline_of(c2.flops, main2, ms2 * n2 * 1e-3, name), "clocks": clk2,
+                            "exp_then_quantize_folded": {"value": c2.flops / (f_ms2 * 1e-3) / 1e12, "ms_per_step": f_ms2,
+                                                         "main_kernel_ms": f_main2, "efq_speedup": f_ms2 / ms2}}
+            del w2
+            torch.cuda.empty_cache()
 
     cpu_baseline = None
     if world == 1 and not args.skip_cpu_baseline:
@@ -496,11 +571,7 @@ def run_cuda(args):
                 "single_stream_ms_per_step": e2e_plain_ms,
                 "single_stream_value": whole_job_tflops(flops, e2e_plain_ms, world)},
         "gpu_launches": 2 * args.steps,     # operand preparation (one kernel for q, k, v) + fused forward
-        "roofline": {"kernel": "attention_fwd_kernel<EFQ>", "bound": "tensor", "achieved": main_tflops, "peak": fp4_peak,
-                     "unit": "TFLOP/s", "frac": main_tflops / fp4_peak, "traffic": traffic,
-                     "peak_source": f"{peaks['source']} bf16 sustained {peaks['bf16_sustained']} TFLOP/s x {NOMINAL_FP4_OVER_BF16} "
-                                    "(nominal FP4:bf16 ratio)", "ms_per_launch": ms_main,
-                     "frac_of_nominal_9pflops": main_tflops / 9000.0},
+        "roofline": roofline,
         "cpu_baseline": cpu_baseline,
         "exp_then_quantize": {"value": flops / (etq_ms_step * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": etq_ms_step,
                               "main_kernel_ms": etq_ms_main, "efq_speedup": etq_ms_step / ms_step},
@@ -512,6 +583,10 @@ def run_cuda(args):
                                      "main_kernel_ms": etqh_ms_main, "efq_speedup": etqh_ms_step / ms_step,
                                      "note": "scale_mode 3: scale_mode 2 with 2 of 8 exponentials by a cubic polynomial on the "
                                              "FMA pipe (takes load off MUFU; does not pay in the fused kernel)"},
+        "exp_then_quantize_fp32_denominator": {"value": flops / (etqd_ms_step * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": etqd_ms_step,
+                                               "main_kernel_ms": etqd_ms_main, "efq_speedup": etqd_ms_step / ms_step,
+                                               "note": "exp-then-quantize whose denominator is the sum of the FP32 exponentials (the convention "
+                                                       "of kernels that quantise P only for the P V product), not the shared operand"},
         "efq_lut": {"value": flops / (lut_ms_step * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": lut_ms_step,
                     "main_kernel_ms": lut_ms_main, "note": "variant 1: 16-level index + folding table (accuracy ablation)"},
         "efq_thresholded_rescale": {"value": flops / (lazy_ms_step * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": lazy_ms_step,
@@ -521,6 +596,7 @@ def run_cuda(args):
         "accuracy": accuracy,
         "stage": stage,
         "microbench": micro,
+        "other_workloads": others,
     }
     print(json.dumps(line))
     if world > 1:
@@ -539,6 +615,8 @@ def main():
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-stage", action="store_true")
     ap.add_argument("--skip-error", action="store_true", help="skip the error-against-exact-attention report")
+    ap.add_argument("--skip-other-workloads", action="store_true",
+                    help="time the named workload only (by default the other two attention shapes follow, a few steps each)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

@@ -142,8 +142,14 @@ efq_status_t efq_attention_fwd(const void* q, const void* k, const void* v, floa
                                const efq_debug_t* debug, void* stream);
 
 /* The MXFP4 comparison path: identical pipeline, the producer replaced by exp-then-quantize
- * (scale_mode as in exp_then_quantize_probgen).  The denominator comes from the same
- * quantised operand as the numerator. */
+ * (scale_mode 0-3 as in exp_then_quantize_probgen).  The denominator comes from the same
+ * quantised operand as the numerator (Eq. denominator-basic applied to the baseline: everything but the
+ * producer held equal).
+ * scale_mode 4 is scale_mode 0 with the other convention for the denominator, the one of attention kernels that
+ * quantise P only for the P V product: l is the sum of the row's FP32 exponentials, carried in registers through
+ * the online recurrence (rescaled with the same alpha), and the ones columns of the tensor-core product are
+ * ignored.  Numerator and denominator then no longer come from one operand; the paper states the shared-operand
+ * rule for its own method only, so both conventions are offered for the baseline. */
 efq_status_t exp_then_quantize_attention_fwd(const void* q, const void* k, const void* v, float* o, int B,
                                              int Hq, int Hkv, int64_t Sq, int64_t Sk, int d, int causal,
                                              float softmax_scale, int scale_mode, void* workspace,
@@ -154,7 +160,8 @@ efq_status_t exp_then_quantize_attention_fwd(const void* q, const void* k, const
  * efq_quantize_qkv: operand preparation only (bf16 -> MXFP4 into the workspace; resets the status word).
  * efq_attention_fwd_quantized: the fused forward on a workspace prepared by efq_quantize_qkv for the
  * same shape; producer 0 = EFQ (with params->variant 1: EFQ-LUT), 1 = exp-then-quantize scale4, 2 = exp-then-quantize
- * scale6, 4 = exp-then-quantize scale4 with the scale folded into the exponential (scale_mode 2), 5 = scale_mode 3.
+ * scale6, 4 = exp-then-quantize scale4 with the scale folded into the exponential (scale_mode 2), 5 = scale_mode 3,
+ * 6 = exp-then-quantize scale4 with the FP32-exponential denominator (scale_mode 4).
  * Arguments, layouts and errors as for efq_attention_fwd. */
 efq_status_t efq_quantize_qkv(const void* q, const void* k, const void* v, int B, int Hq, int Hkv, int64_t Sq,
                               int64_t Sk, int d, void* workspace, size_t workspace_bytes, void* stream);
@@ -305,7 +312,8 @@ efq_status_t efq_attention_fwd_inject_timeout(const void* q, const void* k, cons
 
 const char* efq_status_string(efq_status_t status);
 
-/* Library build tag, e.g. "efq-b200 sm_100a". */
+/* Library build tag: "efq-b200 sm_100a <revision of the fused forward kernel>", e.g. "efq-b200 sm_100a fwd.3".
+ * Measurement records that were taken from a profiler capture name the revision they saw. */
 const char* efq_version(void);
 
 #ifdef __cplusplus

@@ -17,5 +17,5 @@ extern "C" const char* efq_status_string(efq_status_t status)
     return "unknown status";
 }
 
-extern "C" const char* efq_version(void) { return "efq-b200 sm_100a"; }
+extern "C" const char* efq_version(void) { return "efq-b200 sm_100a " EFQ_FWD_KERNEL_REVISION; }
 

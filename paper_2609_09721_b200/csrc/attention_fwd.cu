@@ -72,6 +72,8 @@ struct __align__(1024) Smem {
     uint8_t sf_v[kStages][kSfBytes];
     uint8_t sf_p[2][kSfBytes];
     uint8_t sf_ones[kSfBytes];
+    float lsum_x[2][kTile];   // FP32-denominator baseline only: each group's sum of exponentials ...
+    float mref_x[2][kTile];   // ... and the scaled maximum it refers to
     float runmax[2][kTile];   // running row maximum after the group's latest tile, raw score units
     float alpha[4][kTile];    // [tile mod 4]: rescale factor of the tile, per row (1 where the maximum did not grow)
     uint64_t q_full;
@@ -83,6 +85,7 @@ struct __align__(1024) Smem {
     uint64_t a_bar[4][4];     // [tile mod 4][lane quarter]: alpha of that tile is published
     uint64_t o_ready[2];      // accumulator rows rescaled (or found unchanged) for the tile of this parity
     uint64_t o_done;          // the last P~V of the work item has completed
+    uint64_t l_bar;           // FP32-denominator baseline only: all eight probability warps have written lsum_x / mref_x
     uint32_t tmem_base;
     volatile uint32_t abort_flag;
 };
@@ -170,6 +173,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     if (threadIdx.x == 0) {
         ptx::mbar_init(&sm->q_full, 1);
         ptx::mbar_init(&sm->o_done, 1);
+        ptx::mbar_init(&sm->l_bar, 2 * kGroupWarps);
         for (int s = 0; s < kStages; ++s) {
             ptx::mbar_init(&sm->k_full[s], 1);
             ptx::mbar_init(&sm->k_empty[s], 1);
@@ -361,6 +365,9 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         const int64_t ntile_all = (P.Sk + kTile - 1) / kTile;
         bool ok = true;
         bool in_flight = false;           // the scores of this tile were asked for at the end of the group's previous tile
+        // FP32-denominator baseline (PRODUCER 6): this thread's sum of the row's FP32 exponentials over the group's
+        // own tiles, relative to the scaled maximum m_ref of the latest of them
+        float lsum = 0.0f, m_ref = -INFINITY;
         float r[128];
         const uint32_t s_addr = tmem + lane_base + kColS + 128 * group;
 
@@ -423,13 +430,17 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             // P~V of tile j-2 reads the group's P buffer: asked here, answered while block 0 is computed
             const bool have_p = ptx::mbar_try_wait(&sm->p_empty[sb], ph2 ^ 1u);
 
+            if (PRODUCER == 6) {          // bring the sum to the new reference maximum (two tiles of alpha in one step)
+                if (lsum != 0.0f) lsum *= ex2_approx(__fmul_rn(__fsub_rn(m_ref, m_s), K.LOG2E));
+                m_ref = m_s;
+            }
             // ---- probability operand (Algorithm 1 per block): codes and scales straight into the MMA operand
             uint32_t sfword = 0;
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
                 uint4 codes;
                 uint32_t byte;
-                produce32<PRODUCER, FIX8>(&r[g * 32], bmax[g], m_s, K, codes, byte);
+                produce32<PRODUCER, FIX8>(&r[g * 32], bmax[g], m_s, K, codes, byte, &lsum);
                 if (g == 0 && !have_p) {      // P~V of tile j-2 must have finished: it reads the group's P buffer
                     if (!wait_all(&sm->p_empty[sb], ph2 ^ 1u, sm, P.status)) { ok = false; break; }
                 }
@@ -469,10 +480,17 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         }
         ptx::tmem_wait_ld();              // nothing may be in flight when a bounded wait gave up inside the loop
 
+        if (PRODUCER == 6) {              // both groups' partial denominators meet in shared memory
+            sm->lsum_x[group][row] = lsum;
+            sm->mref_x[group][row] = m_ref;
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&sm->l_bar);
+        }
         // ---- final normalisation O = A / l: each group writes 64 of the 128 channels
         // (a barrier of its own: a group that skipped a phase of the other group's p_empty could not tell
         // an old completion from the last one by parity)
         if (ok) ok = wait_all(&sm->o_done, 0, sm, P.status);
+        if (ok && PRODUCER == 6) ok = wait_all(&sm->l_bar, 0, sm, P.status);
         if (ok) {
             ptx::tc_fence_after_sync();
             uint32_t o[64];
@@ -482,7 +500,15 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             const uint32_t lcol = ptx::tmem_ld1(tmem + lane_base + kColO + 128);
             ptx::tmem_wait_ld();
             if (grow < P.Sq) {
-                const float l = __uint_as_float(lcol);
+                float l = __uint_as_float(lcol);
+                if (PRODUCER == 6) {
+                    // the accumulator refers to the maximum of the last tile, the larger of the two groups' references
+                    const float l0 = sm->lsum_x[0][row], l1 = sm->lsum_x[1][row];
+                    const float m0 = sm->mref_x[0][row], m1 = sm->mref_x[1][row];
+                    const float mf = fmaxf(m0, m1);
+                    l = (l0 != 0.0f ? l0 * ex2_approx(__fmul_rn(__fsub_rn(m0, mf), K.LOG2E)) : 0.0f) +
+                        (l1 != 0.0f ? l1 * ex2_approx(__fmul_rn(__fsub_rn(m1, mf), K.LOG2E)) : 0.0f);
+                }
                 const float inv = l > 0.0f ? 1.0f / l : 0.0f;
                 float4* dst = reinterpret_cast<float4*>(P.o + (bh * P.o_head + grow * P.o_row + 64 * group));
 #pragma unroll
@@ -714,6 +740,7 @@ efq_status_t attention_impl(const void* q, const void* k, const void* v, float* 
         case 3: e = launch_main<3>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
         case 4: e = launch_main<4>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
         case 5: e = launch_main<5>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
+        case 6: e = launch_main<6>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
         default: return EFQ_ERR_INVALID_ARG;
     }
     return e == cudaSuccess ? EFQ_OK : EFQ_ERR_CUDA;
@@ -729,7 +756,8 @@ extern "C" size_t efq_attention_workspace_bytes(int B, int Hq, int Hkv, int64_t 
 }
 
 // Producer ids inside the library: 0 = EFQ (affine rule), 1 / 2 = exp-then-quantize scale4 / scale6, 3 = EFQ-LUT,
-// 4 = exp-then-quantize scale4 with the scale folded into the exponential, 5 = the same with 2 of 8 exponentials by polynomial.
+// 4 = exp-then-quantize scale4 with the scale folded into the exponential, 5 = the same with 2 of 8 exponentials by polynomial,
+// 6 = exp-then-quantize scale4 whose denominator is the sum of the FP32 exponentials (the ones columns are ignored).
 static bool read_params(const efq_params_t* params, float& tau, float& h, bool& lut, float& threshold, efq_status_t& st)
 {
     tau = -3.06f;
@@ -769,7 +797,7 @@ extern "C" efq_status_t exp_then_quantize_attention_fwd(const void* q, const voi
                                                         float softmax_scale, int scale_mode, void* workspace,
                                                         size_t workspace_bytes, const efq_debug_t* debug, void* stream)
 {
-    if (scale_mode < 0 || scale_mode > 3) return EFQ_ERR_INVALID_ARG;
+    if (scale_mode < 0 || scale_mode > 4) return EFQ_ERR_INVALID_ARG;
     return efq::attention_impl(q, k, v, o, B, Hq, Hkv, Sq, Sk, d, causal, softmax_scale, scale_mode >= 2 ? scale_mode + 2 : 1 + scale_mode, 0.0f, 1.0f,
                                workspace, workspace_bytes, debug, static_cast<cudaStream_t>(stream), true, true);
 }
@@ -980,7 +1008,7 @@ extern "C" efq_status_t efq_attention_fwd_varlen(const void* q, const void* k, c
     efq_status_t st;
     if (!read_params(params, tau, h, lut, threshold, st)) return st;
     if (producer == 0 && lut) producer = 3;
-    if (producer < 0 || producer > 5) return EFQ_ERR_INVALID_ARG;
+    if (producer < 0 || producer > 6) return EFQ_ERR_INVALID_ARG;
     const int64_t slot = efq::varlen_slot_bytes(cu_seqlens_q, cu_seqlens_k, n_seqs, Hq, Hkv, d, st);
     if (slot < 0) return st;
     if (n_seqs == 0 || cu_seqlens_q[n_seqs] == 0) return EFQ_OK;     // no query token: nothing to write

@@ -11,6 +11,10 @@ namespace efq {
 
 constexpr int kMxBlock = 32;  // keys per microscaling block
 
+// Revision of the fused forward kernel, part of efq_version().  Raise it whenever attention_fwd_kernel changes:
+// figures copied from a profiler capture (DRAM bytes per launch in the benchmark) are keyed to it.
+#define EFQ_FWD_KERNEL_REVISION "fwd.3"
+
 // Constants of the FP32 code rule, derived on the host in double and rounded once.
 // With x = sigma*r - m_s, k the block's scale exponent and z = x - k ln2 - ln6 (Eq. z-def):
 //   (z - tau) h + 1  =  r*(sigma h) - h m_s - k (h ln2) + (1 - h (ln6 + tau))

@@ -39,7 +39,8 @@ __device__ __forceinline__ float block_max32(const float* r)
 // 32 scores of one microscaling block -> 16 bytes of codes + scale byte.
 // PRODUCER: 0 = EFQ (affine rule), 1 / 2 = exp-then-quantize with the block maximum in [4, 8) / (3, 6],
 // 3 = EFQ-LUT, 4 = exp-then-quantize [4, 8) with the scale folded into the exponential, 5 = the same with 2 of 8
-// exponentials computed by a polynomial on the FMA pipe.
+// exponentials computed by a polynomial on the FMA pipe, 6 = producer 1 that also adds its 32 FP32 exponentials to
+// *psum (for the baseline whose denominator is the sum of the exponentials instead of the quantised operand).
 //
 // EFQ (Algorithm 1), three FMA-pipe instructions per element, bit-identical to
 // c = floor(min(max(fma(r, A, Bb), 0), 7)):
@@ -51,7 +52,7 @@ __device__ __forceinline__ float block_max32(const float* r)
 // only when fma(r, A, Bb) >= 8; FIX8 turns that nibble into 7 (needed when (ln 1.5 - tau) h + 1 can reach 8).
 template <int PRODUCER, bool FIX8>
 __device__ __forceinline__ void produce32(const float* r, float rmax, float m_s, const ProducerConsts& K, uint4& codes,
-                                          uint32_t& byte)
+                                          uint32_t& byte, float* psum = nullptr)
 {
     uint32_t w[4];
     if (PRODUCER == 0) {
@@ -109,20 +110,22 @@ __device__ __forceinline__ void produce32(const float* r, float rmax, float m_s,
         }
     } else {
         float p[32];
-        float amax = 0.0f;
+        float amax = 0.0f, sum = 0.0f;
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
             float x = __fsub_rn(__fmul_rn(K.sigma, r[i]), m_s);
             p[i] = ex2_approx(__fmul_rn(x, K.LOG2E));
             amax = fmaxf(amax, p[i]);
+            if (PRODUCER == 6) sum += p[i];       // masked scores (-inf) give exactly 0
         }
+        if (PRODUCER == 6) *psum += sum;
         if (amax == 0.0f) {
             byte = 0;
             w[0] = w[1] = w[2] = w[3] = 0;
         } else {
             const uint32_t bits = __float_as_uint(amax);
             const int E = static_cast<int>((bits >> 23) & 0xffu) - 127;
-            int e = PRODUCER == 1 ? E - 2 : ((bits & 0x7fffffu) > 0x400000u ? E - 1 : E - 2);
+            int e = (PRODUCER == 1 || PRODUCER == 6) ? E - 2 : ((bits & 0x7fffffu) > 0x400000u ? E - 1 : E - 2);
             e = max(e, -127);
             const float s = __uint_as_float(static_cast<uint32_t>(127 - e) << 23);
             byte = static_cast<uint32_t>(e + 127);

@@ -223,6 +223,36 @@ def test_exp_then_quantize_path(oracle, mode, path):
     print(path, "rel-Frobenius vs exact =", np.linalg.norm(got - exact) / np.linalg.norm(exact))
 
 
+@pytest.mark.parametrize("S,Hq,Hkv,causal,recipe", [(640, 4, 2, True, "k_outliers"), (1000, 2, 1, False, "iid"),
+                                                    (128, 1, 1, True, "iid"), (300, 2, 2, True, "lowrank")])
+def test_exp_then_quantize_with_fp32_denominator(oracle, S, Hq, Hkv, causal, recipe):
+    """scale_mode 4: the quantised operand feeds P~V, the denominator is the sum of the row's FP32 exponentials
+    (the convention of kernels that quantise P for the value product only).  Checked against the oracle's model
+    of that convention; the operand itself is the scale4 producer's (same dump check); and the two conventions
+    differ by more than the tolerance somewhere, so the test tells them apart."""
+    case = inputs.AttentionCase("den", 1, Hq, Hkv, S, S, 128, causal, 500 + S, recipe)
+    (q, k, v), (dq, dk, dv) = _case_tensors(case)
+    head = Hq - 1
+    dump = binding.DebugDump(0, head, 0, S, S)
+    o = binding.exp_then_quantize_attention_fwd(dq, dk, dv, causal, 0.0, 4, debug=dump)
+    o_prod = binding.exp_then_quantize_attention_fwd(dq, dk, dv, causal, 0.0, 4)
+    o_shared = binding.exp_then_quantize_attention_fwd(dq, dk, dv, causal, 0.0, 0)
+    torch.cuda.synchronize()
+    assert torch.equal(o, o_prod)
+    rows = np.array([(0, h, i) for h in range(Hq) for i in range(S)], np.int64)
+    want = oracle.attention_rows(q, k, v, rows, causal, case.softmax_scale, "etq_fp32den")
+    got = o.cpu().numpy().reshape(-1, 128)
+    assert np.abs(got - want).max() <= 5e-3       # device exp is approximate: codes flip at knife-edges
+    _check_dump(oracle, case, dump, _all_rows(case, head, 0, S), MEAN, producer="etq")
+    shared = oracle.attention_rows(q, k, v, rows, causal, case.softmax_scale, "etq")
+    if S >= 300:
+        assert np.abs(want - shared).max() > 2e-2         # the conventions are really different ...
+        assert np.abs(o_shared.cpu().numpy().reshape(-1, 128) - shared).max() <= 5e-3     # ... and each path follows its own
+    exact = oracle.attention_rows(q, k, v, rows, causal, case.softmax_scale, "exact")
+    print("fp32-denominator baseline: rel-Frobenius vs exact =", np.linalg.norm(got - exact) / np.linalg.norm(exact),
+          " shared-operand baseline:", np.linalg.norm(o_shared.cpu().numpy().reshape(-1, 128) - exact) / np.linalg.norm(exact))
+
+
 @pytest.mark.parametrize("causal,producer,params", [(True, 0, None), (False, 0, None), (True, 0, (0.0, 1.0, 1)), (True, 1, None)])
 def test_varlen_packed_batch(oracle, causal, producer, params):
     """Sequences of mixed lengths packed along the token axis: each equals the forward of that sequence alone."""
