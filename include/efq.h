@@ -179,11 +179,20 @@ efq_status_t efq_attention_fwd_quantized(float* o, int B, int Hq, int Hkv, int64
  * sequence sees its keys <= i + len_k - len_q, the rule of efq_attention_fwd); the operands of a sequence are
  * quantised by themselves, so the result of a sequence equals efq_attention_fwd on that sequence alone, bit for
  * bit.  A sequence without queries is skipped; one without keys gets zero rows.  `producer` as for
- * efq_attention_fwd_quantized.  The sequences are launched one after the other on `stream` (two kernels each)
- * and share one workspace slot: efq_attention_varlen_workspace_bytes() gives the size (0 for invalid arguments).
- * Asynchronous; efq_poll_status(workspace, stream) reports the first device-side problem of any sequence.
+ * efq_attention_fwd_quantized.
+ * The whole batch takes two kernel launches on `stream` whatever the number of sequences: one operand preparation
+ * over all sequences (each quantised on its own: V blocks of 32 keys are aligned to the sequence's own key index)
+ * and one fused forward whose work items come from a table in the workspace.  A sequence with so few query tokens
+ * that the query heads of a KV group fit into one 128-row tile (Hq / Hkv * len_q <= 128: decode steps, short
+ * chunks) is run with those heads sharing a tile, so its K/V tiles are read once per KV head.  The same packing is
+ * applied by efq_attention_fwd to a [B, H, S, d] batch with few query tokens; rows never interact, so results do
+ * not depend on it.
+ * The workspace holds the MXFP4 copies of all sequences side by side plus the tables:
+ * efq_attention_varlen_workspace_bytes() gives the size for the given prefix sums (0 for invalid arguments).  The
+ * two prefix arrays are read during the call only.
+ * Asynchronous; efq_poll_status(workspace, stream) reports a device-side problem of any sequence.
  * Errors: INVALID_ARG (null pointer, n_seqs < 0, prefix sums not starting at 0 or decreasing, bad params),
- * UNSUPPORTED (d != 128, a sequence too long for the 32-bit tile coordinates), ALIGNMENT, WORKSPACE, ARCH, CUDA. */
+ * UNSUPPORTED (d != 128, a batch too long for the 32-bit tile coordinates), ALIGNMENT, WORKSPACE, ARCH, CUDA. */
 size_t efq_attention_varlen_workspace_bytes(const int64_t* cu_seqlens_q, const int64_t* cu_seqlens_k, int n_seqs, int Hq,
                                             int Hkv, int d);
 efq_status_t efq_attention_fwd_varlen(const void* q, const void* k, const void* v, float* o, const int64_t* cu_seqlens_q,

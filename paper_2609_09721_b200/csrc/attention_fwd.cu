@@ -30,17 +30,14 @@
 
 #include <mutex>
 
+#include <vector>
+
 #include "efq_common.cuh"
+#include "efq_internal.cuh"
 #include "efq_producers.cuh"
 #include "sm100_ptx.cuh"
 
 namespace efq {
-
-cudaError_t launch_quantize_qkv(const void* q, const void* k, const void* v, int64_t q_heads, int64_t kv_heads, int64_t Sq,
-                                int64_t Sq_pad, int64_t Sk, int64_t Sk_pad, int64_t q_head_stride, int64_t q_row_stride,
-                                int64_t kv_head_stride, int64_t kv_row_stride, uint8_t* q_codes, uint8_t* q_sf,
-                                uint8_t* k_codes, uint8_t* k_sf, uint8_t* vt_codes, uint8_t* v_sf, uint32_t* status,
-                                cudaStream_t stream);
 
 namespace {
 
@@ -103,6 +100,10 @@ struct FwdParams {
     uint32_t* status;
     efq_debug_t dbg;
     int has_dbg;
+    int packed;               // dense batch with few query tokens: the query heads of a KV group share one query tile
+    const SeqDesc* seqs;      // packed variable-length batch: sequence table and one item per CTA (device memory);
+    const ItemDesc* items;    //   NULL for a [B, H, S, d] batch, whose items follow from the block index
+    int64_t v_tiles_per_head; // packed batch: 128-key tiles per KV head in the V^T code matrix (all sequences)
     int inject_skip_loads;    // test hook: the TMA thread loads Q only, so the first wait on K/V runs out
     float rescale_threshold;  // 0: Algorithm 2; > 0: the shifting maximum is kept while the true one is at most this far above
 };
@@ -150,20 +151,50 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
 
-    // ---- work item: heaviest query tiles first, the heads of a GQA group adjacent
-    const int64_t n_qtiles = P.Sq_pad / kTile;
-    const int64_t bh_count = static_cast<int64_t>(P.B) * P.Hq;
-    const int64_t item = blockIdx.x;
-    const int64_t qt = n_qtiles - 1 - item / bh_count;
-    const int64_t bh = item % bh_count;
-    const int b = static_cast<int>(bh / P.Hq);
-    const int hq = static_cast<int>(bh % P.Hq);
-    const int hkv = hq / (P.Hq / P.Hkv);
-    const int64_t q0 = qt * kTile;
-    const int64_t shift = P.Sk - P.Sq;                     // causal: query i sees keys <= i + shift
-    int64_t n_tiles = (P.Sk + kTile - 1) / kTile;
+    // ---- work item.  [B, H, S, d] batch: heaviest query tiles first, the heads of a GQA group adjacent.  Packed
+    // variable-length batch: the item and its sequence come from the tables.  Either way the item is one 128-row
+    // query tile: rows q0 .. q0 + 127 of query head head0, or - "packed", when the sequence has so few query tokens
+    // that the G query heads of a KV group fit into one tile - row r = token r % Sq of query head head0 + r / Sq.
+    const int G = P.Hq / P.Hkv;
+    int64_t Sq, Sk, o_base, q0;
+    int b, head0, hkv, q_row, k_row0, v_x0, v_y0;
+    int64_t sfv_tile0;
+    bool packed;
+    if (P.items != nullptr) {
+        const ItemDesc it = P.items[blockIdx.x];
+        const SeqDesc sd = P.seqs[it.seq];
+        Sq = sd.Sq; Sk = sd.Sk; o_base = sd.o_off; b = it.seq;
+        packed = sd.packed != 0;
+        if (packed) { hkv = it.head; head0 = hkv * G; q0 = 0; q_row = sd.q_row0 + hkv * kTile; }
+        else { head0 = it.head; hkv = head0 / G; q0 = static_cast<int64_t>(it.qt) * kTile; q_row = sd.q_row0 + head0 * sd.Sq_pad + it.qt * kTile; }
+        k_row0 = sd.k_row0 + hkv * sd.Sk_pad;
+        v_x0 = sd.k_col0 / 2;
+        v_y0 = hkv * kTile;
+        sfv_tile0 = static_cast<int64_t>(hkv) * P.v_tiles_per_head + sd.k_col0 / kTile;
+    } else {
+        Sq = P.Sq; Sk = P.Sk;
+        packed = P.packed != 0;
+        const int64_t n_qtiles = packed ? 1 : P.Sq_pad / kTile;
+        const int64_t heads = packed ? P.Hkv : P.Hq;          // heads that own query tiles
+        const int64_t bh_count = static_cast<int64_t>(P.B) * heads;
+        const int64_t item = blockIdx.x;
+        const int64_t qt = n_qtiles - 1 - item / bh_count;
+        const int64_t bh = item % bh_count;
+        b = static_cast<int>(bh / heads);
+        const int hh = static_cast<int>(bh % heads);
+        if (packed) { hkv = hh; head0 = hkv * G; q0 = 0; q_row = static_cast<int>(bh * kTile); }
+        else { head0 = hh; hkv = hh / G; q0 = qt * kTile; q_row = static_cast<int>(bh * P.Sq_pad + q0); }
+        const int64_t kvh = static_cast<int64_t>(b) * P.Hkv + hkv;
+        k_row0 = static_cast<int>(kvh * P.Sk_pad);
+        v_x0 = 0;
+        v_y0 = static_cast<int>(kvh * kTile);
+        sfv_tile0 = kvh * (P.Sk_pad / kTile);
+        o_base = static_cast<int64_t>(b) * P.Hq * P.o_head;
+    }
+    const int64_t shift = Sk - Sq;                         // causal: query i sees keys <= i + shift
+    int64_t n_tiles = (Sk + kTile - 1) / kTile;
     if (P.causal) {
-        int64_t last_row = q0 + kTile - 1 < P.Sq ? q0 + kTile - 1 : P.Sq - 1;
+        int64_t last_row = packed ? Sq - 1 : (q0 + kTile - 1 < Sq ? q0 + kTile - 1 : Sq - 1);
         int64_t last_key = last_row + shift;               // may be negative: nothing visible
         int64_t need = last_key < 0 ? 0 : last_key / kTile + 1;
         if (need < n_tiles) n_tiles = need;
@@ -214,10 +245,9 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     if (run && warp == 0 && lane == 0) {
         // =============================== TMA producer (one thread) ===============================
         ptx::mbar_arrive_expect_tx(&sm->q_full, kTileBytes + kSfBytes);
-        ptx::tma_load_2d(sm->q, &map_q, 0, static_cast<int>(bh * P.Sq_pad + q0), &sm->q_full);
-        ptx::bulk_load_1d(sm->sf_q, P.sf_q + (bh * n_qtiles + qt) * kSfBytes, kSfBytes, &sm->q_full);
-        const int64_t kvh = static_cast<int64_t>(b) * P.Hkv + hkv;
-        const int64_t kv_tiles = P.Sk_pad / kTile;
+        ptx::tma_load_2d(sm->q, &map_q, 0, q_row, &sm->q_full);
+        ptx::bulk_load_1d(sm->sf_q, P.sf_q + static_cast<int64_t>(q_row / kTile) * kSfBytes, kSfBytes, &sm->q_full);
+        const int64_t sfk_tile0 = k_row0 / kTile;
         int s = 0;
         uint32_t ph = 0;
         for (int64_t j = 0; j < (P.inject_skip_loads ? 0 : n_tiles); ++j) {
@@ -225,12 +255,12 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             // looks (S runs ahead) could not tell which completion it sees by parity.
             if (!wait1(&sm->k_empty[s], ph ^ 1u, sm, P.status)) break;
             ptx::mbar_arrive_expect_tx(&sm->k_full[s], kTileBytes + kSfBytes);
-            ptx::tma_load_2d(sm->k[s], &map_k, 0, static_cast<int>(kvh * P.Sk_pad + j * kTile), &sm->k_full[s]);
-            ptx::bulk_load_1d(sm->sf_k[s], P.sf_k + (kvh * kv_tiles + j) * kSfBytes, kSfBytes, &sm->k_full[s]);
+            ptx::tma_load_2d(sm->k[s], &map_k, 0, k_row0 + static_cast<int>(j * kTile), &sm->k_full[s]);
+            ptx::bulk_load_1d(sm->sf_k[s], P.sf_k + (sfk_tile0 + j) * kSfBytes, kSfBytes, &sm->k_full[s]);
             if (!wait1(&sm->v_empty[s], ph ^ 1u, sm, P.status)) break;
             ptx::mbar_arrive_expect_tx(&sm->v_full[s], kTileBytes + kSfBytes);
-            ptx::tma_load_2d(sm->v[s], &map_v, static_cast<int>(j * 64), static_cast<int>(kvh * 128), &sm->v_full[s]);
-            ptx::bulk_load_1d(sm->sf_v[s], P.sf_v + (kvh * kv_tiles + j) * kSfBytes, kSfBytes, &sm->v_full[s]);
+            ptx::tma_load_2d(sm->v[s], &map_v, v_x0 + static_cast<int>(j * 64), v_y0, &sm->v_full[s]);
+            ptx::bulk_load_1d(sm->sf_v[s], P.sf_v + (sfv_tile0 + j) * kSfBytes, kSfBytes, &sm->v_full[s]);
             if (++s == kStages) { s = 0; ph ^= 1u; }
         }
     } else if (run && warp == 1) {
@@ -351,18 +381,32 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     const int quarter = warp & 3;                       // TMEM lane quarter this warp may touch
     const int group = (warp - 4) >> 2;                  // group 0 takes the even KV tiles, group 1 the odd ones
     const uint32_t row = quarter * 32 + lane;           // row inside the query tile: one thread owns one row
-    const int64_t grow = q0 + row;                      // global query row
+    // this thread's query: token index inside the sequence, query head, and whether the row exists
+    int64_t grow;
+    int hq;
+    bool row_valid;
+    if (packed) {
+        const int lq = static_cast<int>(Sq);
+        const int gq = static_cast<int>(row) / lq;
+        grow = static_cast<int>(row) - gq * lq;
+        hq = head0 + gq;
+        row_valid = gq < G;
+    } else {
+        grow = q0 + row;
+        hq = head0;
+        row_valid = grow < Sq;
+    }
     const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
     if (run) {
         // =============================== probability generation ===============================
         const ProducerConsts K = P.K;
-        int64_t limit = P.causal ? grow + shift : P.Sk - 1; // last visible key of this row
-        if (limit > P.Sk - 1) limit = P.Sk - 1;
+        int64_t limit = P.causal ? grow + shift : Sk - 1; // last visible key of this row
+        if (limit > Sk - 1) limit = Sk - 1;
         const bool dbg_row = DEBUG && P.has_dbg && b == P.dbg.batch && hq == P.dbg.head && grow >= P.dbg.q_begin &&
-                             grow < P.dbg.q_end && grow < P.Sq;
+                             grow < P.dbg.q_end && row_valid;
         const int64_t drow = grow - P.dbg.q_begin;
-        const int64_t nblk_all = (P.Sk + 31) / 32;
-        const int64_t ntile_all = (P.Sk + kTile - 1) / kTile;
+        const int64_t nblk_all = (Sk + 31) / 32;
+        const int64_t ntile_all = (Sk + kTile - 1) / kTile;
         bool ok = true;
         bool in_flight = false;           // the scores of this tile were asked for at the end of the group's previous tile
         // FP32-denominator baseline (PRODUCER 6): this thread's sum of the row's FP32 exponentials over the group's
@@ -459,7 +503,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             if (DEBUG && dbg_row) {
                 if (P.dbg.raw_scores) {
                     for (int i = 0; i < 128; ++i)
-                        if (j * kTile + i < P.Sk) P.dbg.raw_scores[drow * P.Sk + j * kTile + i] = r[i];
+                        if (j * kTile + i < Sk) P.dbg.raw_scores[drow * Sk + j * kTile + i] = r[i];
                 }
                 if (P.dbg.row_max) P.dbg.row_max[drow * ntile_all + j] = m_s;
             }
@@ -499,7 +543,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             ptx::tmem_ld32<32>(o_addr + 32, o);
             const uint32_t lcol = ptx::tmem_ld1(tmem + lane_base + kColO + 128);
             ptx::tmem_wait_ld();
-            if (grow < P.Sq) {
+            if (row_valid) {
                 float l = __uint_as_float(lcol);
                 if (PRODUCER == 6) {
                     // the accumulator refers to the maximum of the last tile, the larger of the two groups' references
@@ -510,7 +554,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                         (l1 != 0.0f ? l1 * ex2_approx(__fmul_rn(__fsub_rn(m1, mf), K.LOG2E)) : 0.0f);
                 }
                 const float inv = l > 0.0f ? 1.0f / l : 0.0f;
-                float4* dst = reinterpret_cast<float4*>(P.o + (bh * P.o_head + grow * P.o_row + 64 * group));
+                float4* dst = reinterpret_cast<float4*>(P.o + (o_base + hq * P.o_head + grow * P.o_row + 64 * group));
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
                     float4 v;
@@ -524,8 +568,8 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         }
     } else if (sm->abort_flag == 0) {
         // no visible key for the whole tile: rows are zero
-        if (grow < P.Sq) {
-            float4* dst = reinterpret_cast<float4*>(P.o + (bh * P.o_head + grow * P.o_row + 64 * group));
+        if (row_valid) {
+            float4* dst = reinterpret_cast<float4*>(P.o + (o_base + hq * P.o_head + grow * P.o_row + 64 * group));
             for (int i = 0; i < 16; ++i) dst[i] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
     }
@@ -669,19 +713,53 @@ cudaError_t launch_main(bool debug, bool fix8, dim3 grid, size_t smem, cudaStrea
     }
 }
 
+// The query heads of a KV group share one 128-row query tile when they fit: a decode step (one query token) of a
+// model with 4 query heads per KV head then fills 4 rows of one tile instead of 1 row of each of 4 tiles, and each
+// K/V tile is loaded once per KV head.  Rows are independent of one another on the whole path, so the result is
+// the unpacked one bit for bit.
+bool use_packed_tile(int Hq, int Hkv, int64_t Sq) { return Hq / Hkv > 1 && static_cast<int64_t>(Hq / Hkv) * Sq <= kTile; }
+
+cudaError_t launch_forward(int producer, bool debug, bool fix8, int64_t items, cudaStream_t stream, const CUtensorMap& mq,
+                           const CUtensorMap& mk, const CUtensorMap& mv, const FwdParams& P)
+{
+    if (items <= 0 || items > 0x7fffffffll) return cudaErrorInvalidValue;
+    dim3 grid(static_cast<unsigned>(items));
+    // more than half of the SM's shared memory: one CTA per SM, since each CTA takes all 512 TMEM columns
+    const size_t smem = sizeof(Smem) + 1024 > 120 * 1024 ? sizeof(Smem) + 1024 : 120 * 1024;
+    switch (producer) {
+        case 0: return launch_main<0>(debug, fix8, grid, smem, stream, mq, mk, mv, P);
+        case 1: return launch_main<1>(debug, fix8, grid, smem, stream, mq, mk, mv, P);
+        case 2: return launch_main<2>(debug, fix8, grid, smem, stream, mq, mk, mv, P);
+        case 3: return launch_main<3>(debug, fix8, grid, smem, stream, mq, mk, mv, P);
+        case 4: return launch_main<4>(debug, fix8, grid, smem, stream, mq, mk, mv, P);
+        case 5: return launch_main<5>(debug, fix8, grid, smem, stream, mq, mk, mv, P);
+        case 6: return launch_main<6>(debug, fix8, grid, smem, stream, mq, mk, mv, P);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+// fma(r, A, Bb) can reach 8 only if the residual of a block maximum, below ln 1.5, maps that high
+bool needs_fix8(float tau, float h) { return (log(1.5) - static_cast<double>(tau)) * static_cast<double>(h) + 1.0 > 7.999; }
+
+efq_status_t check_device()
+{
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return EFQ_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return EFQ_ERR_CUDA;
+    return major == 10 ? EFQ_OK : EFQ_ERR_ARCH;
+}
+
 efq_status_t attention_impl(const void* q, const void* k, const void* v, float* o, int B, int Hq, int Hkv, int64_t Sq,
                             int64_t Sk, int d, int causal, float softmax_scale, int producer, float tau, float h,
                             void* workspace, size_t workspace_bytes, const efq_debug_t* debug, cudaStream_t stream,
-                            bool do_quantize, bool do_forward, bool inject_skip_loads = false, float rescale_threshold = 0.0f,
-                            bool token_major = false)
+                            bool do_quantize, bool do_forward, bool inject_skip_loads = false, float rescale_threshold = 0.0f)
 {
-    // token_major: q, k, v are [S, H, d] and o is [Sq, Hq, d] (one sequence of a packed batch; B must be 1);
-    // otherwise [B, H, S, d]
+    // q [B, Hq, Sq, d], k, v [B, Hkv, Sk, d], o [B, Hq, Sq, d]
     if (!q || !k || !v || !o) return EFQ_ERR_INVALID_ARG;
     if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0 || Hq % Hkv != 0) return EFQ_ERR_INVALID_ARG;
-    if (token_major && B != 1) return EFQ_ERR_INVALID_ARG;
     if (d != 128) return EFQ_ERR_UNSUPPORTED;
     if (!shape_ok(B, Hq, Hkv, Sq, Sk, d)) return EFQ_ERR_UNSUPPORTED;
+    if (producer < 0 || producer > 6) return EFQ_ERR_INVALID_ARG;
     if (!(softmax_scale > 0.0f)) softmax_scale = static_cast<float>(1.0 / sqrt(static_cast<double>(d)));
     if (!isfinite(softmax_scale) || !isfinite(tau) || !isfinite(h) || !(h > 0.0f)) return EFQ_ERR_INVALID_ARG;
     auto mis = [](const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0; };
@@ -689,61 +767,112 @@ efq_status_t attention_impl(const void* q, const void* k, const void* v, float* 
     const Workspace w = plan_workspace(B, Hq, Hkv, Sq, Sk);
     if (!workspace || workspace_bytes < w.total) return EFQ_ERR_WORKSPACE;
     if (mis(workspace, 256)) return EFQ_ERR_ALIGNMENT;
-
-    int dev = 0, major = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return EFQ_ERR_CUDA;
-    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return EFQ_ERR_CUDA;
-    if (major != 10) return EFQ_ERR_ARCH;
+    const efq_status_t dev_st = check_device();
+    if (dev_st != EFQ_OK) return dev_st;
 
     uint8_t* ws = static_cast<uint8_t*>(workspace);
+    const bool packed = use_packed_tile(Hq, Hkv, Sq);
+    const int G = Hq / Hkv;
+    const int64_t q_rows = packed ? static_cast<int64_t>(B) * Hkv * kTile : static_cast<int64_t>(B) * Hq * w.Sq_pad;
     if (do_quantize) {
-        const int64_t qh = token_major ? 128 : Sq * 128, qr = token_major ? static_cast<int64_t>(Hq) * 128 : 128;
-        const int64_t kh = token_major ? 128 : Sk * 128, kr = token_major ? static_cast<int64_t>(Hkv) * 128 : 128;
+        QuantSeg sq{}, sk{}, sv{};
+        sq.src = static_cast<const __nv_bfloat16*>(q);
+        sq.heads = packed ? static_cast<int64_t>(B) * Hkv : static_cast<int64_t>(B) * Hq;
+        sq.S = packed ? G * Sq : Sq;
+        sq.S_pad = packed ? kTile : w.Sq_pad;
+        sq.head_stride = Sq * 128; sq.row_stride = 128;
+        sq.pack_lq = packed ? static_cast<int32_t>(Sq) : 0; sq.pack_G = packed ? G : 1;
+        sq.codes = ws + w.qc; sq.sf = ws + w.qsf;
+        sk.src = static_cast<const __nv_bfloat16*>(k);
+        sk.heads = static_cast<int64_t>(B) * Hkv; sk.S = Sk; sk.S_pad = w.Sk_pad;
+        sk.head_stride = Sk * 128; sk.row_stride = 128; sk.pack_G = 1;
+        sk.codes = ws + w.kc; sk.sf = ws + w.ksf;
+        sv = sk;
+        sv.src = static_cast<const __nv_bfloat16*>(v);
+        sv.codes = ws + w.vt; sv.sf = ws + w.vsf;
+        sv.v_row_bytes = w.Sk_pad / 2; sv.v_x0 = 0; sv.v_sf_tiles_per_head = w.Sk_pad / kTile; sv.v_sf_tile0 = 0;
         // one launch for the three operands; it also clears the status words the forward starts from
-        if (launch_quantize_qkv(q, k, v, static_cast<int64_t>(B) * Hq, static_cast<int64_t>(B) * Hkv, Sq, w.Sq_pad, Sk,
-                                w.Sk_pad, qh, qr, kh, kr, ws + w.qc, ws + w.qsf, ws + w.kc, ws + w.ksf, ws + w.vt,
-                                ws + w.vsf, reinterpret_cast<uint32_t*>(ws + w.status), stream) != cudaSuccess)
-            return EFQ_ERR_CUDA;
+        if (launch_quantize_qkv(sq, sk, sv, reinterpret_cast<uint32_t*>(ws + w.status), stream) != cudaSuccess) return EFQ_ERR_CUDA;
     }
     if (!do_forward) return EFQ_OK;
 
     CUtensorMap mq, mk, mv;
-    if (!encode_map(&mq, ws + w.qc, 64, static_cast<uint64_t>(B) * Hq * w.Sq_pad)) return EFQ_ERR_CUDA;
+    if (!encode_map(&mq, ws + w.qc, 64, static_cast<uint64_t>(q_rows))) return EFQ_ERR_CUDA;
     if (!encode_map(&mk, ws + w.kc, 64, static_cast<uint64_t>(B) * Hkv * w.Sk_pad)) return EFQ_ERR_CUDA;
     if (!encode_map(&mv, ws + w.vt, static_cast<uint64_t>(w.Sk_pad / 2), static_cast<uint64_t>(B) * Hkv * 128)) return EFQ_ERR_CUDA;
 
-    FwdParams P;
+    FwdParams P{};
     P.B = B; P.Hq = Hq; P.Hkv = Hkv; P.Sq = Sq; P.Sk = Sk; P.Sq_pad = w.Sq_pad; P.Sk_pad = w.Sk_pad;
     P.causal = causal ? 1 : 0;
     P.K = producer == 3 ? make_producer_consts_lut(softmax_scale) : make_producer_consts(softmax_scale, tau, h);
     P.sf_q = ws + w.qsf; P.sf_k = ws + w.ksf; P.sf_v = ws + w.vsf;
     P.o = o;
-    P.o_head = token_major ? 128 : Sq * 128;
-    P.o_row = token_major ? static_cast<int64_t>(Hq) * 128 : 128;
+    P.o_head = Sq * 128;
+    P.o_row = 128;
     P.status = reinterpret_cast<uint32_t*>(ws + w.status);
+    P.packed = packed ? 1 : 0;
+    P.seqs = nullptr; P.items = nullptr; P.v_tiles_per_head = 0;
     P.inject_skip_loads = inject_skip_loads ? 1 : 0;
     P.rescale_threshold = rescale_threshold;
     P.has_dbg = debug ? 1 : 0;
     if (debug) P.dbg = *debug; else P.dbg = efq_debug_t{};
 
-    const int64_t items = (w.Sq_pad / kTile) * B * Hq;
-    dim3 grid(static_cast<unsigned>(items));
-    // more than half of the SM's shared memory: one CTA per SM, since each CTA takes all 512 TMEM columns
-    const size_t smem = sizeof(Smem) + 1024 > 120 * 1024 ? sizeof(Smem) + 1024 : 120 * 1024;
-    // fma(r, A, Bb) can reach 8 only if the residual of a block maximum, below ln 1.5, maps that high
-    const bool fix8 = (log(1.5) - static_cast<double>(tau)) * static_cast<double>(h) + 1.0 > 7.999;
-    cudaError_t e;
-    switch (producer) {
-        case 0: e = launch_main<0>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
-        case 1: e = launch_main<1>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
-        case 2: e = launch_main<2>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
-        case 3: e = launch_main<3>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
-        case 4: e = launch_main<4>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
-        case 5: e = launch_main<5>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
-        case 6: e = launch_main<6>(debug != nullptr, fix8, grid, smem, stream, mq, mk, mv, P); break;
-        default: return EFQ_ERR_INVALID_ARG;
+    const int64_t items = packed ? static_cast<int64_t>(B) * Hkv : (w.Sq_pad / kTile) * B * Hq;
+    return launch_forward(producer, debug != nullptr, needs_fix8(tau, h), items, stream, mq, mk, mv, P) == cudaSuccess ? EFQ_OK
+                                                                                                                  : EFQ_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Packed variable-length batch: every sequence quantised by itself, all of them in two launches
+// ------------------------------------------------------------------------------------------------
+// Workspace: status words | tables (sequence table, item table, quantiser jobs, their CTA prefix sums) |
+// Q codes [rows of all sequences, 64 B] | Q scale tiles | K codes | K scale tiles |
+// V^T codes [Hkv * 128, sum of Sk_pad / 2 B] (the sequences side by side along the keys) | V scale tiles.
+struct VarlenPlan {
+    int n_active;                    // sequences with query and key tokens
+    int64_t q_rows, k_rows, k_cols;  // rows of the Q and K code matrices, keys along V^T (all padded to 128)
+    int64_t items, quant_ctas;
+    size_t tables, seqs_off, items_off, jobs_off, prefix_off, qc, qsf, kc, ksf, vt, vsf, total;
+};
+
+// checks the two prefix arrays and lays the workspace out; false with st set on bad input
+bool plan_varlen(const int64_t* cu_q, const int64_t* cu_k, int n_seqs, int Hq, int Hkv, int d, VarlenPlan& p, efq_status_t& st)
+{
+    st = EFQ_OK;
+    if (!cu_q || !cu_k || n_seqs < 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0) { st = EFQ_ERR_INVALID_ARG; return false; }
+    if (d != 128) { st = EFQ_ERR_UNSUPPORTED; return false; }
+    if (n_seqs > 0 && (cu_q[0] != 0 || cu_k[0] != 0)) { st = EFQ_ERR_INVALID_ARG; return false; }
+    p = VarlenPlan{};
+    for (int s = 0; s < n_seqs; ++s) {
+        const int64_t lq = cu_q[s + 1] - cu_q[s], lk = cu_k[s + 1] - cu_k[s];
+        if (lq < 0 || lk < 0) { st = EFQ_ERR_INVALID_ARG; return false; }
+        if (lq == 0 || lk == 0) continue;
+        const bool packed = use_packed_tile(Hq, Hkv, lq);
+        const int64_t lq_pad = packed ? kTile : (lq + kTile - 1) / kTile * kTile, lk_pad = (lk + kTile - 1) / kTile * kTile;
+        ++p.n_active;
+        p.q_rows += (packed ? Hkv : Hq) * lq_pad;
+        p.k_rows += Hkv * lk_pad;
+        p.k_cols += lk_pad;
+        p.items += packed ? Hkv : (lq_pad / kTile) * Hq;
+        p.quant_ctas += ((packed ? Hkv : Hq) * lq_pad * 4 + 255) / 256 + (Hkv * lk_pad * 4 + 255) / 256 + (Hkv * (lk_pad / 32) + 1) / 2;
     }
-    return e == cudaSuccess ? EFQ_OK : EFQ_ERR_CUDA;
+    // 32-bit tile coordinates and grid sizes
+    if (p.q_rows >= (1ll << 31) || p.k_rows >= (1ll << 31) || p.k_cols >= (1ll << 31) || p.items >= (1ll << 31) ||
+        p.quant_ctas >= (1ll << 31)) { st = EFQ_ERR_UNSUPPORTED; return false; }
+    size_t off = 1024;
+    p.seqs_off = off;   off = align_up(off + sizeof(SeqDesc) * p.n_active, 256);
+    p.items_off = off;  off = align_up(off + sizeof(ItemDesc) * static_cast<size_t>(p.items), 256);
+    p.jobs_off = off;   off = align_up(off + sizeof(QuantJob) * 3 * p.n_active, 256);
+    p.prefix_off = off; off = align_up(off + sizeof(int32_t) * (3 * p.n_active + 1), 1024);
+    p.tables = off - 1024;
+    p.qc = off;  off = align_up(off + static_cast<size_t>(p.q_rows) * 64, 1024);
+    p.qsf = off; off = align_up(off + static_cast<size_t>(p.q_rows / kTile) * kSfBytes, 1024);
+    p.kc = off;  off = align_up(off + static_cast<size_t>(p.k_rows) * 64, 1024);
+    p.ksf = off; off = align_up(off + static_cast<size_t>(p.k_rows / kTile) * kSfBytes, 1024);
+    p.vt = off;  off = align_up(off + static_cast<size_t>(Hkv) * 128 * (p.k_cols / 2), 1024);
+    p.vsf = off; off = align_up(off + static_cast<size_t>(Hkv) * (p.k_cols / kTile) * kSfBytes, 1024);
+    p.total = off;
+    return true;
 }
 
 }  // namespace
@@ -966,35 +1095,13 @@ extern "C" efq_status_t efq_attention_fwd_host_pipelined(const void* q_host, con
 // ------------------------------------------------------------------------------------------------
 // Packed variable-length batch: the sequences of the batch lie one after the other along the token axis
 // ------------------------------------------------------------------------------------------------
-namespace efq {
-namespace {
-// checks the two prefix arrays and returns the workspace slot of the largest sequence (0: nothing to do; -1: bad input)
-int64_t varlen_slot_bytes(const int64_t* cu_q, const int64_t* cu_k, int n_seqs, int Hq, int Hkv, int d, efq_status_t& st)
-{
-    st = EFQ_OK;
-    if (!cu_q || !cu_k || n_seqs < 0 || Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0) { st = EFQ_ERR_INVALID_ARG; return -1; }
-    if (d != 128) { st = EFQ_ERR_UNSUPPORTED; return -1; }
-    if (n_seqs > 0 && (cu_q[0] != 0 || cu_k[0] != 0)) { st = EFQ_ERR_INVALID_ARG; return -1; }
-    size_t slot = 0;
-    for (int s = 0; s < n_seqs; ++s) {
-        const int64_t lq = cu_q[s + 1] - cu_q[s], lk = cu_k[s + 1] - cu_k[s];
-        if (lq < 0 || lk < 0) { st = EFQ_ERR_INVALID_ARG; return -1; }
-        if (lq == 0 || lk == 0) continue;
-        if (!shape_ok(1, Hq, Hkv, lq, lk, d)) { st = EFQ_ERR_UNSUPPORTED; return -1; }
-        const size_t need = plan_workspace(1, Hq, Hkv, lq, lk).total;
-        if (need > slot) slot = need;
-    }
-    return static_cast<int64_t>(slot);
-}
-}  // namespace
-}  // namespace efq
-
 extern "C" size_t efq_attention_varlen_workspace_bytes(const int64_t* cu_seqlens_q, const int64_t* cu_seqlens_k, int n_seqs,
                                                        int Hq, int Hkv, int d)
 {
     efq_status_t st;
-    const int64_t slot = efq::varlen_slot_bytes(cu_seqlens_q, cu_seqlens_k, n_seqs, Hq, Hkv, d, st);
-    return slot < 0 ? 0 : static_cast<size_t>(slot) + 1024;
+    efq::VarlenPlan p;
+    if (!efq::plan_varlen(cu_seqlens_q, cu_seqlens_k, n_seqs, Hq, Hkv, d, p, st)) return 0;
+    return p.total;
 }
 
 extern "C" efq_status_t efq_attention_fwd_varlen(const void* q, const void* k, const void* v, float* o,
@@ -1003,43 +1110,123 @@ extern "C" efq_status_t efq_attention_fwd_varlen(const void* q, const void* k, c
                                                  const efq_params_t* params, void* workspace, size_t workspace_bytes,
                                                  void* stream)
 {
+    using namespace efq;
     float tau, h, threshold;
     bool lut;
     efq_status_t st;
     if (!read_params(params, tau, h, lut, threshold, st)) return st;
     if (producer == 0 && lut) producer = 3;
     if (producer < 0 || producer > 6) return EFQ_ERR_INVALID_ARG;
-    const int64_t slot = efq::varlen_slot_bytes(cu_seqlens_q, cu_seqlens_k, n_seqs, Hq, Hkv, d, st);
-    if (slot < 0) return st;
+    VarlenPlan p;
+    if (!plan_varlen(cu_seqlens_q, cu_seqlens_k, n_seqs, Hq, Hkv, d, p, st)) return st;
     if (n_seqs == 0 || cu_seqlens_q[n_seqs] == 0) return EFQ_OK;     // no query token: nothing to write
     if (!q || !k || !v || !o) return EFQ_ERR_INVALID_ARG;
-    if (!workspace || workspace_bytes < static_cast<size_t>(slot) + 1024) return EFQ_ERR_WORKSPACE;
+    if (!(softmax_scale > 0.0f)) softmax_scale = static_cast<float>(1.0 / sqrt(static_cast<double>(d)));
+    if (!isfinite(softmax_scale) || !isfinite(tau) || !isfinite(h) || !(h > 0.0f)) return EFQ_ERR_INVALID_ARG;
+    auto mis = [](const void* ptr, uintptr_t a) { return (reinterpret_cast<uintptr_t>(ptr) & (a - 1)) != 0; };
+    if (mis(q, 16) || mis(k, 16) || mis(v, 16) || mis(o, 16)) return EFQ_ERR_ALIGNMENT;
+    if (!workspace || workspace_bytes < p.total) return EFQ_ERR_WORKSPACE;
+    if (mis(workspace, 256)) return EFQ_ERR_ALIGNMENT;
+    const efq_status_t dev_st = check_device();
+    if (dev_st != EFQ_OK) return dev_st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     uint8_t* ws = static_cast<uint8_t*>(workspace);
-    uint32_t* agg = reinterpret_cast<uint32_t*>(ws + slot);          // first problem seen by any sequence
-    if (cudaMemsetAsync(agg, 0, 4, s) != cudaSuccess) return EFQ_ERR_CUDA;
-    if (cudaMemsetAsync(ws, 0, 4, s) != cudaSuccess) return EFQ_ERR_CUDA;
+    const int G = Hq / Hkv;
+
+    // host copies of the tables, in the layout of the workspace's table region
+    std::vector<uint8_t> tables(p.tables, 0);
+    SeqDesc* seqs = reinterpret_cast<SeqDesc*>(tables.data() + (p.seqs_off - 1024));
+    ItemDesc* items = reinterpret_cast<ItemDesc*>(tables.data() + (p.items_off - 1024));
+    QuantJob* jobs = reinterpret_cast<QuantJob*>(tables.data() + (p.jobs_off - 1024));
+    int32_t* prefix = reinterpret_cast<int32_t*>(tables.data() + (p.prefix_off - 1024));
+    const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q);
+    const __nv_bfloat16* kb = static_cast<const __nv_bfloat16*>(k);
+    const __nv_bfloat16* vb = static_cast<const __nv_bfloat16*>(v);
+    int64_t q_row = 0, k_row = 0, k_col = 0, n_items = 0, ctas = 0;
+    int a = 0;
     for (int i = 0; i < n_seqs; ++i) {
         const int64_t q0 = cu_seqlens_q[i], k0 = cu_seqlens_k[i];
         const int64_t lq = cu_seqlens_q[i + 1] - q0, lk = cu_seqlens_k[i + 1] - k0;
         if (lq == 0) continue;
-        float* oi = o + q0 * Hq * 128;
         if (lk == 0) {               // no key at all: the rows are zero, as for a causal row that sees nothing
-            if (cudaMemsetAsync(oi, 0, static_cast<size_t>(lq) * Hq * 128 * sizeof(float), s) != cudaSuccess) return EFQ_ERR_CUDA;
+            if (cudaMemsetAsync(o + q0 * Hq * 128, 0, static_cast<size_t>(lq) * Hq * 128 * sizeof(float), s) != cudaSuccess) return EFQ_ERR_CUDA;
             continue;
         }
-        const uint16_t* qi = static_cast<const uint16_t*>(q) + q0 * Hq * 128;
-        const uint16_t* ki = static_cast<const uint16_t*>(k) + k0 * Hkv * 128;
-        const uint16_t* vi = static_cast<const uint16_t*>(v) + k0 * Hkv * 128;
-        // the sequences run in stream order, so one workspace slot serves them all
-        st = efq::attention_impl(qi, ki, vi, oi, 1, Hq, Hkv, lq, lk, d, causal, softmax_scale, producer, tau, h, ws,
-                                 static_cast<size_t>(slot), nullptr, s, true, true, false, threshold, true);
-        if (st != EFQ_OK) return st;
-        efq::merge_status_kernel<<<1, 1, 0, s>>>(agg, reinterpret_cast<const uint32_t*>(ws), 0);
-        if (cudaGetLastError() != cudaSuccess) return EFQ_ERR_CUDA;
+        const bool packed = use_packed_tile(Hq, Hkv, lq);
+        const int64_t lq_pad = packed ? kTile : (lq + kTile - 1) / kTile * kTile, lk_pad = (lk + kTile - 1) / kTile * kTile;
+        SeqDesc& sd = seqs[a];
+        sd.Sq = lq; sd.Sk = lk; sd.o_off = q0 * Hq * 128;
+        sd.q_row0 = static_cast<int32_t>(q_row); sd.Sq_pad = static_cast<int32_t>(lq_pad);
+        sd.k_row0 = static_cast<int32_t>(k_row); sd.Sk_pad = static_cast<int32_t>(lk_pad);
+        sd.k_col0 = static_cast<int32_t>(k_col); sd.packed = packed ? 1 : 0;
+        // work items: heaviest query tiles of a sequence first, the heads of a GQA group adjacent
+        if (packed) {
+            for (int hk = 0; hk < Hkv; ++hk) items[n_items++] = ItemDesc{a, 0, hk, 0};
+        } else {
+            for (int64_t qt = lq_pad / kTile - 1; qt >= 0; --qt)
+                for (int hh = 0; hh < Hq; ++hh) items[n_items++] = ItemDesc{a, static_cast<int32_t>(qt), hh, 0};
+        }
+        // quantiser jobs: the sequence's own Q, K, V (token-major source: a head is 128 elements, a token H * 128)
+        QuantJob& jq = jobs[3 * a];
+        QuantJob& jk = jobs[3 * a + 1];
+        QuantJob& jv = jobs[3 * a + 2];
+        jq.kind = kQuantRows; jk.kind = kQuantRows; jv.kind = kQuantV;
+        jq.seg.src = qb + q0 * Hq * 128;
+        jq.seg.heads = packed ? Hkv : Hq; jq.seg.S = packed ? G * lq : lq; jq.seg.S_pad = lq_pad;
+        jq.seg.head_stride = 128; jq.seg.row_stride = static_cast<int64_t>(Hq) * 128;
+        jq.seg.pack_lq = packed ? static_cast<int32_t>(lq) : 0; jq.seg.pack_G = packed ? G : 1;
+        jq.seg.codes = ws + p.qc + q_row * 64; jq.seg.sf = ws + p.qsf + (q_row / kTile) * kSfBytes;
+        jk.seg.src = kb + k0 * Hkv * 128;
+        jk.seg.heads = Hkv; jk.seg.S = lk; jk.seg.S_pad = lk_pad;
+        jk.seg.head_stride = 128; jk.seg.row_stride = static_cast<int64_t>(Hkv) * 128; jk.seg.pack_G = 1;
+        jk.seg.codes = ws + p.kc + k_row * 64; jk.seg.sf = ws + p.ksf + (k_row / kTile) * kSfBytes;
+        jv.seg = jk.seg;
+        jv.seg.src = vb + k0 * Hkv * 128;
+        jv.seg.codes = ws + p.vt; jv.seg.sf = ws + p.vsf;
+        jv.seg.v_row_bytes = p.k_cols / 2; jv.seg.v_x0 = k_col / 2;
+        jv.seg.v_sf_tiles_per_head = p.k_cols / kTile; jv.seg.v_sf_tile0 = k_col / kTile;
+        for (int t = 0; t < 3; ++t) {
+            prefix[3 * a + t] = static_cast<int32_t>(ctas);
+            ctas += quantize_job_ctas(jobs[3 * a + t]);
+        }
+        q_row += (packed ? Hkv : Hq) * lq_pad;
+        k_row += Hkv * lk_pad;
+        k_col += lk_pad;
+        ++a;
     }
-    efq::merge_status_kernel<<<1, 1, 0, s>>>(reinterpret_cast<uint32_t*>(ws), agg, 1);
-    return cudaGetLastError() == cudaSuccess ? EFQ_OK : EFQ_ERR_CUDA;
+    if (p.n_active == 0)             // nothing to launch: the status word still has to read "no problem"
+        return cudaMemsetAsync(ws, 0, 4, s) == cudaSuccess ? EFQ_OK : EFQ_ERR_CUDA;
+    prefix[3 * p.n_active] = static_cast<int32_t>(ctas);
+
+    // Pageable host memory: the call returns once the bytes sit in the driver's staging area, so the vector may go.
+    if (cudaMemcpyAsync(ws + 1024, tables.data(), p.tables, cudaMemcpyHostToDevice, s) != cudaSuccess) return EFQ_ERR_CUDA;
+    if (launch_quantize_jobs(reinterpret_cast<const QuantJob*>(ws + p.jobs_off), reinterpret_cast<const int32_t*>(ws + p.prefix_off),
+                             3 * p.n_active, ctas, reinterpret_cast<uint32_t*>(ws), s) != cudaSuccess)
+        return EFQ_ERR_CUDA;
+
+    CUtensorMap mq, mk, mv;
+    if (!encode_map(&mq, ws + p.qc, 64, static_cast<uint64_t>(p.q_rows))) return EFQ_ERR_CUDA;
+    if (!encode_map(&mk, ws + p.kc, 64, static_cast<uint64_t>(p.k_rows))) return EFQ_ERR_CUDA;
+    if (!encode_map(&mv, ws + p.vt, static_cast<uint64_t>(p.k_cols / 2), static_cast<uint64_t>(Hkv) * 128)) return EFQ_ERR_CUDA;
+
+    FwdParams P{};
+    P.B = p.n_active; P.Hq = Hq; P.Hkv = Hkv; P.Sq = 0; P.Sk = 0; P.Sq_pad = 0; P.Sk_pad = 0;
+    P.causal = causal ? 1 : 0;
+    P.K = producer == 3 ? make_producer_consts_lut(softmax_scale) : make_producer_consts(softmax_scale, tau, h);
+    P.sf_q = ws + p.qsf; P.sf_k = ws + p.ksf; P.sf_v = ws + p.vsf;
+    P.o = o;
+    P.o_head = 128;                                   // token-major: a head is 128 elements, a token Hq * 128
+    P.o_row = static_cast<int64_t>(Hq) * 128;
+    P.status = reinterpret_cast<uint32_t*>(ws);
+    P.packed = 0;
+    P.seqs = reinterpret_cast<const SeqDesc*>(ws + p.seqs_off);
+    P.items = reinterpret_cast<const ItemDesc*>(ws + p.items_off);
+    P.v_tiles_per_head = p.k_cols / kTile;
+    P.inject_skip_loads = 0;
+    P.rescale_threshold = threshold;
+    P.has_dbg = 0;
+    P.dbg = efq_debug_t{};
+    return launch_forward(producer, false, needs_fix8(tau, h), n_items, s, mq, mk, mv, P) == cudaSuccess ? EFQ_OK : EFQ_ERR_CUDA;
 }
 
 extern "C" efq_status_t efq_poll_status(void* workspace, void* stream)

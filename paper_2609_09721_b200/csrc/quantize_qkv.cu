@@ -8,13 +8,16 @@
 //
 // Layouts written (S_pad = S rounded up to 128; padding rows/keys are zero codes, byte 0):
 //   Q, K codes   [B*H, S_pad, 64 B]          row-major, 2 codes per byte, element 2u in the low nibble
+//                (few query tokens: the query heads of a KV group packed into one 128-row tile, [B*Hkv, 128, 64 B])
 //   V^T codes    [B*Hkv, 128 (channel), S_pad/2 B]   keys contiguous: the P~V contraction runs over keys
+//                (packed variable-length batch: [Hkv, 128, sum of S_pad / 2 B], the sequences side by side along the keys)
 //   scale tiles  one 512-byte tile per 128 rows (Q, K: rows = tokens, 4 blocks along d;
 //                V: rows = channels, 4 key blocks of the 128-key tile); byte of (row r, block b) at
 //                (r % 32) * 16 + (r / 32) * 4 + b, the order the scale-factor copy into TMEM expects.
 #include <cuda_bf16.h>
 
 #include "efq_common.cuh"
+#include "efq_internal.cuh"
 
 namespace efq {
 
@@ -56,22 +59,28 @@ __device__ __forceinline__ void mxfp4_block(const uint32_t (&w)[16], uint4& code
 
 __device__ __forceinline__ uint32_t sf_tile_offset(uint32_t r, uint32_t b) { return (r & 31u) * 16u + (r >> 5) * 4u + b; }
 
-// One thread per (row, 32-wide block along d); d = 128.  The input is addressed by strides in elements:
-// element (head, row, c) at x[head * head_stride + row * row_stride + c].  The four scale bytes of a row are
-// gathered by shuffles and stored as one word by the thread of block 0.
-__device__ __forceinline__ void quantize_row_block(const __nv_bfloat16* __restrict__ x, int64_t t, int64_t S,
-                                                   int64_t S_pad, int64_t head_stride, int64_t row_stride,
-                                                   uint8_t* __restrict__ codes, uint8_t* __restrict__ sf, bool active)
+// One thread per (row, 32-wide block along d); d = 128.  t counts (padded row, block) pairs of the job.  The four
+// scale bytes of a row are gathered by shuffles and stored as one word by the thread of block 0.
+template <bool DENSE>
+__device__ __forceinline__ void quantize_row_block(const QuantSeg& g, int64_t t)
 {
+    const bool active = t < g.heads * g.S_pad * 4;
     const int blk = static_cast<int>(t & 3);
-    const int64_t prow = t >> 2;               // padded row index over all heads
+    const int64_t prow = t >> 2;               // padded row index over all heads of the job
     uint4 c = make_uint4(0, 0, 0, 0);
     uint32_t byte = 0;
     if (active) {
-        const int64_t head = prow / S_pad;
-        const int64_t row = prow - head * S_pad;
-        if (row < S) {
-            const uint4* src = reinterpret_cast<const uint4*>(x + head * head_stride + row * row_stride + blk * 32);
+        const int64_t head = prow / g.S_pad;
+        const int64_t row = prow - head * g.S_pad;
+        if (row < g.S) {
+            int64_t src_head = head, src_row = row;
+            if (g.pack_G > 1) {                // packed query tile: rows run over (query head of the group, token)
+                const int64_t gq = row / g.pack_lq;
+                src_head = head * g.pack_G + gq;
+                src_row = row - gq * g.pack_lq;
+            }
+            const uint4* src = reinterpret_cast<const uint4*>(g.src + src_head * g.head_stride +
+                                                              src_row * (DENSE ? 128 : g.row_stride) + blk * 32);
             uint32_t w[16];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -80,7 +89,7 @@ __device__ __forceinline__ void quantize_row_block(const __nv_bfloat16* __restri
             }
             mxfp4_block(w, c, byte);
         }
-        *reinterpret_cast<uint4*>(codes + prow * 64 + blk * 16) = c;
+        *reinterpret_cast<uint4*>(g.codes + prow * 64 + blk * 16) = c;
     }
     // lanes 4k .. 4k+3 hold the four blocks of one row (the thread count is a multiple of 4, so a row never
     // straddles warps or the end of the range)
@@ -90,40 +99,39 @@ __device__ __forceinline__ void quantize_row_block(const __nv_bfloat16* __restri
     word |= __shfl_down_sync(0xffffffffu, byte, 3) << 24;
     if (active && blk == 0) {
         const int64_t tile = prow >> 7;        // S_pad is a multiple of 128, so tiles never straddle heads
-        *reinterpret_cast<uint32_t*>(sf + tile * 512 + sf_tile_offset(static_cast<uint32_t>(prow & 127), 0)) = word;
+        *reinterpret_cast<uint32_t*>(g.sf + tile * 512 + sf_tile_offset(static_cast<uint32_t>(prow & 127), 0)) = word;
     }
 }
 
-// One thread per (32-key block, channel); consecutive threads take consecutive channels.
-__device__ __forceinline__ void quantize_v_block(const __nv_bfloat16* __restrict__ v, int64_t kb, int ch, int64_t S,
-                                                 int64_t S_pad, int64_t head_stride, int64_t row_stride,
-                                                 uint8_t* __restrict__ vt_codes, uint8_t* __restrict__ sf)
+// One thread per (32-key block, channel); consecutive threads take consecutive channels.  kb counts the key blocks
+// of the job over all heads.
+template <bool DENSE>
+__device__ __forceinline__ void quantize_v_block(const QuantSeg& g, int64_t kb, int ch)
 {
-    const int64_t blocks_per_head = S_pad / 32;
+    const int64_t blocks_per_head = g.S_pad / 32;
+    if (kb >= g.heads * blocks_per_head) return;
     const int64_t head = kb / blocks_per_head;
     const int64_t kblk = kb - head * blocks_per_head;
-    const uint16_t* src = reinterpret_cast<const uint16_t*>(v) + head * head_stride + kblk * 32 * row_stride + ch;
+    const int64_t rs = DENSE ? 128 : g.row_stride;
+    const uint16_t* src = reinterpret_cast<const uint16_t*>(g.src) + head * g.head_stride + kblk * 32 * rs + ch;
     uint32_t w[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
         const int64_t k0 = kblk * 32 + 2 * i;
-        uint32_t lo = k0 < S ? __ldg(src + (2 * i) * row_stride) : 0u;
-        uint32_t hi = k0 + 1 < S ? __ldg(src + (2 * i + 1) * row_stride) : 0u;
+        uint32_t lo = k0 < g.S ? __ldg(src + (2 * i) * rs) : 0u;
+        uint32_t hi = k0 + 1 < g.S ? __ldg(src + (2 * i + 1) * rs) : 0u;
         w[i] = lo | (hi << 16);
     }
     uint4 c;
     uint32_t byte;
     mxfp4_block(w, c, byte);
-    *reinterpret_cast<uint4*>(vt_codes + (head * 128 + ch) * (S_pad / 2) + kblk * 16) = c;
-    const int64_t tile = head * (S_pad / 128) + (kblk >> 2);
-    sf[tile * 512 + sf_tile_offset(static_cast<uint32_t>(ch), static_cast<uint32_t>(kblk & 3))] = static_cast<uint8_t>(byte);
+    *reinterpret_cast<uint4*>(g.codes + (head * 128 + ch) * g.v_row_bytes + g.v_x0 + kblk * 16) = c;
+    const int64_t tile = head * g.v_sf_tiles_per_head + g.v_sf_tile0 + (kblk >> 2);
+    g.sf[tile * 512 + sf_tile_offset(static_cast<uint32_t>(ch), static_cast<uint32_t>(kblk & 3))] = static_cast<uint8_t>(byte);
 }
 
 struct QuantArgs {
-    const __nv_bfloat16 *q, *k, *v;
-    int64_t q_heads, kv_heads, Sq, Sq_pad, Sk, Sk_pad;
-    int64_t q_head_stride, q_row_stride, kv_head_stride, kv_row_stride;     // elements
-    uint8_t *q_codes, *q_sf, *k_codes, *k_sf, *vt_codes, *v_sf;
+    QuantSeg q, k, v;
     uint32_t* status;           // 256 words, cleared here: the forward that follows starts from a clean status
     int64_t q_ctas, k_ctas;     // the grid: Q rows, then K rows, then V key blocks (two per CTA)
 };
@@ -135,43 +143,59 @@ __global__ void __launch_bounds__(256) quantize_qkv_kernel(const QuantArgs a)
     const int64_t cta = blockIdx.x;
     if (cta == 0) a.status[threadIdx.x] = 0u;
     if (cta < a.q_ctas) {
-        const int64_t t = cta * 256 + threadIdx.x;
-        quantize_row_block(a.q, t, a.Sq, a.Sq_pad, a.q_head_stride, DENSE ? 128 : a.q_row_stride, a.q_codes, a.q_sf,
-                           t < a.q_heads * a.Sq_pad * 4);
+        quantize_row_block<DENSE>(a.q, cta * 256 + threadIdx.x);
     } else if (cta < a.q_ctas + a.k_ctas) {
-        const int64_t t = (cta - a.q_ctas) * 256 + threadIdx.x;
-        quantize_row_block(a.k, t, a.Sk, a.Sk_pad, a.kv_head_stride, DENSE ? 128 : a.kv_row_stride, a.k_codes, a.k_sf,
-                           t < a.kv_heads * a.Sk_pad * 4);
+        quantize_row_block<DENSE>(a.k, (cta - a.q_ctas) * 256 + threadIdx.x);
     } else {
-        const int64_t kb = (cta - a.q_ctas - a.k_ctas) * 2 + (threadIdx.x >> 7);
-        if (kb < a.kv_heads * (a.Sk_pad / 32))
-            quantize_v_block(a.v, kb, static_cast<int>(threadIdx.x & 127), a.Sk, a.Sk_pad, a.kv_head_stride,
-                             DENSE ? 128 : a.kv_row_stride, a.vt_codes, a.v_sf);
+        quantize_v_block<DENSE>(a.v, (cta - a.q_ctas - a.k_ctas) * 2 + (threadIdx.x >> 7), static_cast<int>(threadIdx.x & 127));
     }
 }
 
-cudaError_t launch_quantize_qkv(const void* q, const void* k, const void* v, int64_t q_heads, int64_t kv_heads, int64_t Sq,
-                                int64_t Sq_pad, int64_t Sk, int64_t Sk_pad, int64_t q_head_stride, int64_t q_row_stride,
-                                int64_t kv_head_stride, int64_t kv_row_stride, uint8_t* q_codes, uint8_t* q_sf,
-                                uint8_t* k_codes, uint8_t* k_sf, uint8_t* vt_codes, uint8_t* v_sf, uint32_t* status,
-                                cudaStream_t stream)
+// The jobs of a packed batch in one launch: a CTA finds its job by bisection of the prefix sums.
+__global__ void __launch_bounds__(256) quantize_jobs_kernel(const QuantJob* __restrict__ jobs, const int32_t* __restrict__ first_cta,
+                                                            int n_jobs, uint32_t* status)
+{
+    const int cta = blockIdx.x;
+    if (cta == 0) status[threadIdx.x] = 0u;
+    int lo = 0, hi = n_jobs;                  // first_cta[lo] <= cta < first_cta[hi]
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(first_cta + mid) <= cta) lo = mid; else hi = mid;
+    }
+    const QuantJob& job = jobs[lo];
+    const int64_t local = cta - __ldg(first_cta + lo);
+    if (job.kind == kQuantRows) quantize_row_block<false>(job.seg, local * 256 + threadIdx.x);
+    else quantize_v_block<false>(job.seg, local * 2 + (threadIdx.x >> 7), static_cast<int>(threadIdx.x & 127));
+}
+
+int64_t quantize_job_ctas(const QuantJob& job)
+{
+    if (job.kind == kQuantRows) return (job.seg.heads * job.seg.S_pad * 4 + 255) / 256;
+    return (job.seg.heads * (job.seg.S_pad / 32) + 1) / 2;
+}
+
+cudaError_t launch_quantize_qkv(const QuantSeg& q, const QuantSeg& k, const QuantSeg& v, uint32_t* status, cudaStream_t stream)
 {
     QuantArgs a;
-    a.q = static_cast<const __nv_bfloat16*>(q); a.k = static_cast<const __nv_bfloat16*>(k); a.v = static_cast<const __nv_bfloat16*>(v);
-    a.q_heads = q_heads; a.kv_heads = kv_heads; a.Sq = Sq; a.Sq_pad = Sq_pad; a.Sk = Sk; a.Sk_pad = Sk_pad;
-    a.q_head_stride = q_head_stride; a.q_row_stride = q_row_stride;
-    a.kv_head_stride = kv_head_stride; a.kv_row_stride = kv_row_stride;
-    a.q_codes = q_codes; a.q_sf = q_sf; a.k_codes = k_codes; a.k_sf = k_sf; a.vt_codes = vt_codes; a.v_sf = v_sf;
+    a.q = q; a.k = k; a.v = v;
     a.status = status;
-    a.q_ctas = (q_heads * Sq_pad * 4 + 255) / 256;
-    a.k_ctas = (kv_heads * Sk_pad * 4 + 255) / 256;
-    const int64_t v_ctas = (kv_heads * (Sk_pad / 32) + 1) / 2;
+    a.q_ctas = (q.heads * q.S_pad * 4 + 255) / 256;
+    a.k_ctas = (k.heads * k.S_pad * 4 + 255) / 256;
+    const int64_t v_ctas = (v.heads * (v.S_pad / 32) + 1) / 2;
     const int64_t grid = a.q_ctas + a.k_ctas + v_ctas;
     if (grid <= 0 || grid > 0x7fffffffll) return cudaErrorInvalidValue;
-    if (q_row_stride == 128 && kv_row_stride == 128)
+    if (q.row_stride == 128 && k.row_stride == 128 && v.row_stride == 128)
         quantize_qkv_kernel<true><<<static_cast<unsigned>(grid), 256, 0, stream>>>(a);
     else
         quantize_qkv_kernel<false><<<static_cast<unsigned>(grid), 256, 0, stream>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_quantize_jobs(const QuantJob* jobs, const int32_t* first_cta, int n_jobs, int64_t total_ctas, uint32_t* status,
+                                 cudaStream_t stream)
+{
+    if (n_jobs <= 0 || total_ctas <= 0 || total_ctas > 0x7fffffffll) return cudaErrorInvalidValue;
+    quantize_jobs_kernel<<<static_cast<unsigned>(total_ctas), 256, 0, stream>>>(jobs, first_cta, n_jobs, status);
     return cudaGetLastError();
 }
 

@@ -294,6 +294,63 @@ def test_varlen_packed_batch(oracle, causal, producer, params):
         assert err <= (TOL_O if producer == 0 else 5e-3)
 
 
+def test_varlen_decode_batch_of_64_sequences(oracle):
+    """A decode step over 64 sequences of mixed context lengths (one query token each, 8 query / 2 KV heads): the
+    whole batch goes through one operand-preparation launch and one fused launch, the four query heads of a KV
+    group sharing a query tile.  Every sequence equals the forward of that sequence alone bit for bit; a few are
+    checked against the oracle."""
+    Hq, Hkv = 8, 2
+    rng = np.random.default_rng(5)
+    lens = [(1, int(n)) for n in rng.integers(40, 3000, 64)]
+    lens[7] = (1, 128)
+    lens[9] = (1, 1)
+    lens[11] = (3, 777)          # a short chunk of query tokens, still packed (4 heads x 3 tokens)
+    qs, ks, vs, alone = [], [], [], []
+    for n, (lq, lk) in enumerate(lens):
+        case = inputs.AttentionCase("d", 1, Hq, Hkv, lq, lk, 128, True, 900 + n, "k_outliers")
+        (q, k, v), (dq, dk, dv) = _case_tensors(case)
+        qs.append(dq[0].permute(1, 0, 2))
+        ks.append(dk[0].permute(1, 0, 2))
+        vs.append(dv[0].permute(1, 0, 2))
+        alone.append((case, (q, k, v), (dq, dk, dv)))
+    qp, kp, vp = (torch.cat(t, 0).contiguous() for t in (qs, ks, vs))
+    cu_q = np.concatenate([[0], np.cumsum([a for a, _ in lens])])
+    cu_k = np.concatenate([[0], np.cumsum([b for _, b in lens])])
+    o = binding.efq_attention_fwd_varlen(qp, kp, vp, cu_q, cu_k, True)
+    torch.cuda.synchronize()
+    for n, (lq, lk) in enumerate(lens):
+        case, (q, k, v), (dq, dk, dv) = alone[n]
+        one = binding.efq_attention_fwd(dq, dk, dv, True)
+        got = o[cu_q[n]:cu_q[n + 1]].permute(1, 0, 2)
+        assert torch.equal(got, one[0]), f"sequence {n}"
+        if n in (0, 7, 9, 11, 40):
+            rows = np.array([(0, h, i) for h in range(Hq) for i in range(lq)], np.int64)
+            want = oracle.attention_rows(q, k, v, rows, True, case.softmax_scale, "efq")
+            assert np.abs(got.reshape(-1, 128).cpu().numpy() - want).max() <= TOL_O
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,Sq,Sk,causal", [(3, 8, 2, 1, 1000, True), (2, 4, 1, 32, 300, True), (1, 6, 2, 40, 129, False)])
+def test_packed_query_tile_of_a_dense_batch(oracle, B, Hq, Hkv, Sq, Sk, causal):
+    """Few query tokens in a [B, H, S, d] batch: the query heads of a KV group share one query tile.  The result is
+    checked against the oracle on every row and, with the dump of one head, on the operand bits."""
+    case = inputs.AttentionCase("pk", B, Hq, Hkv, Sq, Sk, 128, causal, 640 + Sq, "k_outliers")
+    (q, k, v), (dq, dk, dv) = _case_tensors(case)
+    head = Hq - 2
+    dump = binding.DebugDump(B - 1, head, 0, Sq, Sk)
+    o = binding.efq_attention_fwd(dq, dk, dv, causal, 0.0, None, debug=dump)
+    o_prod = binding.efq_attention_fwd(dq, dk, dv, causal, 0.0, None)
+    torch.cuda.synchronize()
+    assert torch.equal(o, o_prod)
+    rows = np.array([(b, h, i) for b in range(B) for h in range(Hq) for i in range(Sq)], np.int64)
+    want = oracle.attention_rows(q, k, v, rows, causal, case.softmax_scale, "efq")
+    assert np.abs(o.cpu().numpy().reshape(-1, 128) - want).max() <= TOL_O
+    # the dump belongs to batch entry B - 1: compare with the oracle's dump of those rows
+    drows = np.array([(B - 1, head, i) for i in range(Sq)], np.int64)
+    _, wd = oracle.attention_rows(q, k, v, drows, causal, case.softmax_scale, "efq", dumps=True)
+    assert np.array_equal(dump.codes.cpu().numpy(), wd["codes"])
+    assert np.array_equal(dump.scales.cpu().numpy(), wd["scales"])
+
+
 def test_varlen_argument_errors():
     q = torch.zeros((8, 2, 128), dtype=torch.bfloat16, device="cuda")
     good = [0, 8]
