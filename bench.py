@@ -40,7 +40,7 @@ FALLBACK_HBM_GBS = 6650.0
 # from the single-pass ncu capture summarised in the named profile, and valid only for the kernel revision that
 # capture saw (the library's version tag); for any other revision the line carries null.
 NCU_DRAM_BYTES_PER_LAUNCH = {
-    "qwen3_8b_16k": {"bytes": 57208832 + 217094144, "kernel_revision": "fwd.3", "profile": "profiles/attention_fwd_qwen3_8b_16k.md"},
+    "qwen3_8b_16k": {"bytes": 57717248 + 217710080, "kernel_revision": "fwd.3", "profile": "profiles/attention_fwd_qwen3_8b_16k.md"},
 }
 BURST_REGION_S = 1.0   # a timed region shorter than this runs at burst clocks: its roofline uses the burst peak
 
